@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the batched SPDY dynamic program.
+
+One "step" = one pass of the whole path (forward dynamic program, final minimum over the budget
+axis, walk back) over one batch of synthetic candidates.  The default workload is the
+BERT-base-shaped search (L 72, K 42, B 10000, N 4096 candidates per GPU).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+prints one JSON line on rank 0.  `--impl reference` times the CPU oracle on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+SM_COUNT_NOMINAL = 148
+SM_MAX_MHZ_NOMINAL = 1965.0
+CELLS_PER_CLK_PER_SM = 32.0  # one 4-byte shared-memory read per cell update, 32 banks x 4 B per clock
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload config 1..4 (default 2: BERT-base shape)")
+    ap.add_argument("--n", type=int, default=None, help="candidates per GPU (default: the config's)")
+    ap.add_argument("--budget", type=int, default=None, help="override B (config 4 sweep)")
+    ap.add_argument("--table", default="default", choices=["default", "arg", "row"])
+    ap.add_argument("--threads", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU work budget of the oracle legs")
+    return ap.parse_args()
+
+
+def host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.05):
+        self.index, self.period = index, period
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self.error = None
+
+    def _run(self):
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            uuid = None
+            try:
+                import torch
+
+                uuid = str(torch.cuda.get_device_properties(self.index).uuid)
+            except Exception:
+                pass
+            h = None
+            if uuid:
+                for cand in (f"GPU-{uuid}", uuid):
+                    try:
+                        h = pynvml.nvmlDeviceGetHandleByUUID(cand.encode() if isinstance(cand, str) else cand)
+                        break
+                    except Exception:
+                        h = None
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            names = {
+                pynvml.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                pynvml.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                pynvml.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                pynvml.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+                pynvml.nvmlClocksThrottleReasonHwPowerBrakeSlowdown: "hw_power_brake",
+            }
+            while not self._stop.is_set():
+                self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                mask = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                time.sleep(self.period)
+        except Exception as exc:  # NVML missing: report it, never fail the bench
+            self.error = repr(exc)
+
+    def __enter__(self):
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thread.join(timeout=2.0)
+
+    def summary(self) -> dict:
+        out = {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+               "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        if self.error:
+            out["error"] = self.error
+        return out
+
+
+def oracle_baseline(wl, cpu_seconds: float) -> dict:
+    """The oracle as it stands on the host cores, on a bounded prefix of the same candidates."""
+    import oracle
+
+    cores = host_cores()
+    t0 = time.perf_counter()
+    oracle.solve_batch(wl.errors[:1], wl.times, wl.B, threads=1)
+    t_one = max(time.perf_counter() - t0, 1e-6)
+    n = int(min(wl.N, max(cores, cpu_seconds * cores / t_one)))
+    threads = min(cores, n)
+    t0 = time.perf_counter()
+    oracle.solve_batch(wl.errors[:n], wl.times, wl.B, threads=threads)
+    dt = time.perf_counter() - t0
+    return {"value": n / dt, "unit": "candidates/s", "cores": threads, "kind": "oracle",
+            "sample": f"first {n} of {wl.N} candidates of {wl.name}, one single-threaded solver per core",
+            "single_core_ms_per_candidate": 1e3 * t_one, "seconds": dt}
+
+
+def run_reference(args):
+    """CPU oracle as the reference arm; rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2201_13096_b200 import workloads as W
+    import oracle
+
+    cores = host_cores()
+    wl = W.make_workload(args.config, N=args.n, B=args.budget)
+    t0 = time.perf_counter()
+    oracle.solve_batch(wl.errors[:1], wl.times, wl.B, threads=1)
+    t_one = max(time.perf_counter() - t0, 1e-6)
+    total_steps = args.steps + args.warmup
+    per_step_s = min(20.0, 150.0 / max(total_steps, 1))
+    n = int(min(wl.N, max(cores, per_step_s * cores / t_one)))
+    threads = min(cores, n)
+    for _ in range(args.warmup):
+        oracle.solve_batch(wl.errors[:n], wl.times, wl.B, threads=threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.solve_batch(wl.errors[:n], wl.times, wl.B, threads=threads)
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = f"each step solves the first {n} of {wl.N} candidates of {wl.name}"
+    line = {
+        "impl": "reference", "metric": "candidate_profiles_per_s", "value": value, "unit": "candidates/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "L": wl.L, "K": wl.K, "B": wl.B, "candidates_per_step": n},
+        "nominal_cell_updates_per_s": value * wl.L * wl.K * wl.B,
+        "cpu_baseline": {"value": value, "unit": "candidates/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "candidates/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2201_13096_b200 import binding, workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the solver has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    # Candidates are independent problems: every rank solves its own shard of one long candidate
+    # stream against the same timing table; no data-path collective.
+    probe = W.make_workload(args.config, N=1, B=args.budget)
+    n_per_rank = args.n if args.n is not None else {1: 1024, 2: 4096, 3: 1024, 4: 4096}[args.config]
+    wl = W.make_workload(args.config, N=n_per_rank, B=args.budget, start=rank * n_per_rank)
+    assert np.array_equal(probe.times, wl.times)
+    fmt = {"default": 0, "arg": 1, "row": 2}[args.table]
+    plan = binding.Plan(wl.times, wl.B, device=local_rank, table_format=fmt, threads=args.threads)
+    info = plan.info
+    plan.enable_timing(True)
+
+    errors = torch.from_numpy(wl.errors).to(dev)
+    profile = torch.empty((wl.N, wl.L), dtype=torch.uint8, device=dev)
+    cost = torch.empty(wl.N, dtype=torch.float32, device=dev)
+    time_used = torch.empty(wl.N, dtype=torch.int32, device=dev)
+    ws_bytes = min(plan.workspace_bytes(wl.N), 48 << 30)
+    workspace = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
+    waves = -(-plan.workspace_bytes(wl.N) // max(ws_bytes, 1)) if info["feasible"] else 1
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)  # > 126 MB L2
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.solve_batch(plan, errors, profile, cost, time_used, workspace, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 0)):
+        flush.fill_(1)
+        step()
+    barrier()
+    plan.check_status()
+
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    fwd_ms, back_ms = [], []
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        for i in range(args.steps):
+            flush.fill_(i & 0xFF)  # evict L2 between timed steps (outside the event pair)
+            starts[i].record(stream)
+            step()
+            stops[i].record(stream)
+            f, b = plan.last_timing()  # waits for this step
+            fwd_ms.append(f)
+            back_ms.append(b)
+        barrier()
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
+    total_ms = float(sum(step_ms))
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    plan.check_status()
+
+    # End to end through the host-buffer entry point: pinned host inputs, copies inside the timing.
+    e2e = None
+    if not args.no_e2e:
+        h_err = torch.from_numpy(wl.errors).pin_memory()
+        h_prof = torch.empty((wl.N, wl.L), dtype=torch.uint8).pin_memory()
+        h_cost = torch.empty(wl.N, dtype=torch.float32).pin_memory()
+        h_time = torch.empty(wl.N, dtype=torch.int32).pin_memory()
+        for _ in range(2):
+            binding.solve_batch_host(plan, h_err, h_prof, h_cost, h_time, stream)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            binding.solve_batch_host(plan, h_err, h_prof, h_cost, h_time, stream)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        same = (torch.equal(h_prof, profile.cpu()) and torch.equal(h_time, time_used.cpu())
+                and h_cost.numpy().tobytes() == cost.cpu().numpy().tobytes())
+        if not same:
+            raise SystemExit("host-buffer path disagrees with the device-buffer path")
+        e2e = {"value": world * wl.N * args.steps / e2e_s, "unit": "candidates/s",
+               "h2d_bytes_per_step": int(h_err.numel() * 4),
+               "d2h_bytes_per_step": int(wl.N * (wl.L + 8)), "ms_per_step": 1e3 * e2e_s / args.steps}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = total_ms / args.steps
+    cand_per_s = world * wl.N / (ms_per_step * 1e-3)
+    fwd = float(np.mean(fwd_ms))
+    back = float(np.mean(back_ms))
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    sm_max = float(peaks.get("sm_max_mhz", SM_MAX_MHZ_NOMINAL))
+    peak_cells = info["sm_count"] * sm_max * 1e6 * CELLS_PER_CLK_PER_SM
+    useful = info["useful_updates"] * wl.N  # per launch (one wave = whole batch unless split)
+    achieved = useful / waves / (fwd / waves * 1e-3) if fwd > 0 else 0.0
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    cellb = 4 if info["table_format"] == 2 else 1
+    hbm_bytes = wl.N * (info["band_cells"] * cellb + wl.L * wl.K * 4)
+    line = {
+        "metric": "candidate_profiles_per_s", "value": cand_per_s, "unit": "candidates/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "L": wl.L, "K": wl.K, "B": wl.B, "candidates_per_gpu": wl.N,
+                   "l2": "256 MiB buffer rewritten between timed steps (L2 flush); the walk-back table "
+                         f"written per step is {info['table_bytes_per_candidate'] * wl.N / 1e6:.0f} MB",
+                   "timing": "sum of per-step CUDA-event pairs on the launch stream, max over ranks",
+                   "table_format": {1: "arg_u8", 2: "row_f32"}[info["table_format"]],
+                   "threads": info["threads"], "ctas_per_sm": info["ctas_per_sm"], "span": info["span"],
+                   "waves": int(waves)},
+        "nominal_cell_updates_per_s": cand_per_s * info["nominal_updates"],
+        "useful_cell_updates_per_s": cand_per_s * info["useful_updates"],
+        "roofline": {
+            "bound": "alu", "kernel": "spdy_forward_kernel",
+            "achieved": achieved / 1e9, "peak": peak_cells / 1e9, "unit": "Gcell-updates/s",
+            "frac": achieved / peak_cells, "traffic": None,
+            "peak_is": f"{info['sm_count']} SMs x {sm_max:.0f} MHz x 32 four-byte shared-memory reads per clock "
+                       "(one read per cell update); of nominal unit counts, max clock of measured",
+            "kernel_ms": fwd, "walkback_ms": back,
+            "useful_updates_per_launch": useful / waves, "issued_updates_per_launch": info["issued_updates"] * wl.N / waves,
+        },
+        "roofline_hbm": {"bound": "hbm", "achieved": hbm_bytes / (fwd * 1e-3) / 1e9 if fwd > 0 else 0.0,
+                         "peak": hbm_peak, "unit": "GB/s",
+                         "frac": (hbm_bytes / (fwd * 1e-3) / 1e9 / hbm_peak) if fwd > 0 else 0.0,
+                         "note": "secondary: table writes + error reads of the forward kernel, of measured copy bandwidth"},
+        "gpu_launches": int(2 * waves * args.steps),
+        "clocks": clocks.summary(),
+    }
+    if e2e:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = oracle_baseline(wl, args.cpu_seconds)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,181 @@
+/*
+ * spdy_dp.h - C ABI of the batched SPDY dynamic program for NVIDIA B200 (sm_100a).
+ *
+ * The problem (Frantar & Alistarh, "SPDY: Accurate Pruning with Speedup Guarantees",
+ * Section 3.1, Eq. 1): for each of L layers pick one of K choices so that the summed error is
+ * minimal while the summed (integer, bucketed) time stays within a budget B.  Section 3.2
+ * (Eq. 2-3) gives the exact dynamic program over "lowest error of the first l layers taking
+ * exactly t buckets"; Appendix A (Algorithm 1) adds the choice table and the walk back from the
+ * last layer that recovers the profile.  This library solves N such problems at once - the N
+ * candidate error tables one step of the search of Section 3.3 / Algorithm 4 proposes - that
+ * share one timing table.
+ *
+ * Semantics fixed here (bit-exact, fp32, round-to-nearest, one add per cell):
+ *   D_0[0] = +0, D_0[t>0] = +inf;
+ *   D_l[t] = min over k (ascending, strict "<": lowest k wins ties) of D_{l-1}[t - times[l][k]]
+ *            + errors[n][l][k], over the choices with times[l][k] <= t;
+ *   t*     = lowest t in [0, B] minimising D_L[t];   cost = D_L[t*];   time_used = t*;
+ *   profile[l] = the winning k along the walk back from (L, t*).
+ * A candidate with no profile of finite error inside the budget is not an error: it gets
+ * cost = +inf, time_used = -1 and profile bytes 0xFF.
+ *
+ * Value domain: errors may be any finite fp32 or +inf (a choice that must not be taken);
+ * NaN and -inf are invalid (results unspecified, no fault).  times are >= 0, may be 0, may repeat
+ * and may exceed B (such a choice is unusable).  1 <= K <= 255, L >= 1, B >= 0, N >= 0.
+ *
+ * All functions return SPDY_OK (0) or a negative spdy_status; none throws, aborts or traps.
+ * "host" / "device" below says where a pointer must point.  The library keeps no caller
+ * pointer beyond the stream work it enqueued.
+ */
+#ifndef SPDY_DP_H
+#define SPDY_DP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum spdy_status {
+    SPDY_OK = 0,
+    SPDY_ERR_INVALID_ARG = -1,        /* null pointer, size out of range, negative time, bad alignment */
+    SPDY_ERR_WORKSPACE_TOO_SMALL = -2, /* workspace cannot hold even one candidate's table */
+    SPDY_ERR_UNSUPPORTED = -3,        /* rows too wide for the largest launch shape on this device */
+    SPDY_ERR_CUDA = -4,               /* a CUDA runtime call failed; see spdy_last_cuda_error() */
+    SPDY_ERR_NO_MEMORY = -5,          /* host or device allocation failed */
+    SPDY_ERR_INTERNAL = -6            /* a self-check inside the kernels failed */
+} spdy_status;
+
+/* What the forward kernel stores per live cell for the walk back (Algorithm 1's matrix P). */
+typedef enum spdy_table_format {
+    SPDY_TABLE_DEFAULT = 0, /* let the plan choose (currently SPDY_TABLE_ARG_U8) */
+    SPDY_TABLE_ARG_U8 = 1,  /* the winning choice index, one byte per cell (Algorithm 1's P) */
+    SPDY_TABLE_ROW_F32 = 2  /* the row value D_l[t], 4 bytes per cell; the walk back re-derives
+                               the lowest winning k with the same fp32 add (identical results) */
+} spdy_table_format;
+
+typedef struct spdy_options {
+    int32_t table_format;  /* spdy_table_format */
+    int32_t threads;       /* threads per CTA, 0 = choose; multiple of 32 in [64, 1024] */
+    int32_t cluster;       /* CTAs cooperating on one candidate, 0 = choose; 1, 2, 4 or 8 */
+    int32_t reserved[5];   /* must be 0 */
+} spdy_options;
+
+/* Facts about a plan: shapes, the launch shape chosen, and work counts for measurement. */
+typedef struct spdy_plan_info {
+    int32_t L, K, B;
+    int32_t feasible;       /* 0: sum of per-layer minimum times exceeds B, every candidate is infeasible */
+    int32_t max_width;      /* widest live band, in cells */
+    int32_t span;           /* cells one warp processes per pass */
+    int32_t threads;        /* threads per CTA */
+    int32_t cluster;        /* CTAs per candidate */
+    int32_t table_format;   /* resolved spdy_table_format */
+    int32_t ctas_per_sm;    /* resident CTAs per SM the launch shape allows */
+    int32_t sm_count;
+    int32_t reserved0;
+    int64_t smem_bytes;     /* dynamic shared memory per CTA */
+    int64_t table_bytes_per_candidate; /* walk-back table bytes one candidate needs */
+    int64_t band_cells;     /* sum over layers of the live band width (cells written per candidate) */
+    int64_t useful_updates; /* sum over (layer, choice) of cells whose source lies in the previous band */
+    int64_t issued_updates; /* cell updates the kernel actually issues per candidate (span granularity) */
+    int64_t nominal_updates;/* L*K*B per candidate, the unit of the headline metric */
+} spdy_plan_info;
+
+typedef struct spdy_plan spdy_plan; /* opaque; owns only its own small host and device tables */
+
+/*
+ * Build a plan for one timing table and budget (Eq. 1's constraint; the live band of each DP
+ * row follows from the per-layer minimum and maximum times).  Synchronous; small host work plus
+ * one small host-to-device copy on `device`.
+ *   times_host  host, [L][K] int32 row-major, read during the call only.
+ *   device      CUDA device ordinal, or -1 for a host-only plan (info queries only; solving
+ *               with it returns SPDY_ERR_INVALID_ARG).
+ *   opts        host, may be NULL for defaults.
+ *   *out        receives the plan; destroy with spdy_plan_destroy.
+ * Errors: INVALID_ARG (null, L<1, K<1, K>255, B<0, a negative time, bad option), UNSUPPORTED
+ * (band too wide for the device's shared memory at the largest cluster), NO_MEMORY, CUDA.
+ */
+int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int32_t K, int32_t B,
+                     int device, const spdy_options *opts);
+void spdy_plan_destroy(spdy_plan *plan);
+
+/* Fill *info (host).  INVALID_ARG on null. */
+int spdy_plan_get_info(const spdy_plan *plan, spdy_plan_info *info);
+
+/* Per-layer live band [lo, lo+width) of row l (l = 1..L stored at index l-1); host arrays of L
+ * int32 each, either may be NULL.  For an infeasible plan widths are 0. */
+int spdy_plan_get_bands(const spdy_plan *plan, int32_t *lo_host, int32_t *width_host);
+
+/* Bytes of workspace that let N candidates run as a single wave.  Any workspace of at least
+ * spdy_workspace_bytes(plan, 1) is accepted; a smaller-than-full one makes the batch run as
+ * several waves on the stream.  Returns 0 for a null plan or N <= 0. */
+size_t spdy_workspace_bytes(const spdy_plan *plan, int64_t N);
+
+/*
+ * Solve N candidates (Eq. 2-3 forward, final min over t <= B, walk back of Algorithm 1).
+ * Asynchronous: enqueues kernels on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
+ * default stream) and returns; outputs are valid once the stream reaches that point.
+ *   errors_dev     device, [N][L][K] fp32 row-major, 4-byte aligned.
+ *   profile_dev    device, [N][L] uint8 out: choice index per layer (0xFF.. if infeasible).
+ *   cost_dev       device, [N] fp32 out.
+ *   time_used_dev  device, [N] int32 out (-1 if infeasible).
+ *   workspace_dev  device, caller-owned scratch of workspace_bytes bytes, 256-byte aligned;
+ *                  contents undefined afterwards; must not be shared by solves that overlap.
+ * Errors: INVALID_ARG, WORKSPACE_TOO_SMALL, CUDA (launch failure).
+ */
+int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
+                     uint8_t *profile_dev, float *cost_dev, int32_t *time_used_dev,
+                     void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Same computation with HOST buffers (pageable or pinned): copies errors to the device, solves,
+ * copies the three outputs back and waits for the stream.  Device staging memory is owned by
+ * the plan and grows on demand (cudaMalloc on first use or growth), so one plan must not run
+ * two host-buffer solves at the same time.
+ */
+int spdy_solve_batch_host(spdy_plan *plan, const float *errors_host, int64_t N,
+                          uint8_t *profile_host, float *cost_host, int32_t *time_used_host,
+                          void *cuda_stream);
+
+/*
+ * One-shot form of the whole path: errors[N][L][K], times[L][K], budget B -> profile, cost,
+ * time_used, all device pointers on the current device except nothing else.  Reads times back to
+ * the host, builds a transient plan, allocates and frees its own workspace, and waits for the
+ * stream before returning (synchronous).  Convenience for callers that solve once.
+ */
+int spdy_solve_batch_simple(const float *errors_dev, const int32_t *times_dev, int64_t N,
+                            int32_t L, int32_t K, int32_t B, uint8_t *profile_dev, float *cost_dev,
+                            int32_t *time_used_dev, void *cuda_stream);
+
+/*
+ * Read and clear the plan's device-side self-check word: the walk-back kernels set it if a table
+ * entry is not a valid choice or the walk does not end at t = 0 (which would mean corrupted
+ * scratch or invalid inputs such as NaN).  Waits for `cuda_stream`.  Returns SPDY_OK,
+ * SPDY_ERR_INTERNAL if the word was set, or a CUDA error.
+ */
+int spdy_plan_check_status(spdy_plan *plan, void *cuda_stream);
+
+/*
+ * Measurement aid.  With timing on, every spdy_solve_batch on this plan records CUDA events on
+ * the solve's stream around the forward kernel(s) and around the walk-back kernel(s);
+ * spdy_plan_last_timing waits for the last solve's events and returns the summed durations in
+ * milliseconds (either pointer may be NULL).  Off by default; adds three event records per wave.
+ * A plan with timing on must not run solves concurrently from several host threads.
+ */
+int spdy_plan_enable_timing(spdy_plan *plan, int on);
+int spdy_plan_last_timing(spdy_plan *plan, float *forward_ms_host, float *walkback_ms_host);
+
+/* Static, human-readable text for a status code. */
+const char *spdy_strerror(int status);
+
+/* The cudaError_t value of the most recent failed CUDA call on this host thread (0 if none). */
+int spdy_last_cuda_error(void);
+
+/* Library version, major*1000 + minor. */
+int spdy_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPDY_DP_H */

@@ -1,0 +1,240 @@
+"""Thin ctypes binding of ``include/spdy_dp.h``: argument marshalling only.
+
+Every step of the path (forward dynamic program, final minimum, walk back) runs in the CUDA
+library; PyTorch supplies device buffers and the stream.  There is no CPU fallback: if the
+library has not been built the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libspdy_dp.so")
+
+SPDY_TABLE_DEFAULT, SPDY_TABLE_ARG_U8, SPDY_TABLE_ROW_F32 = 0, 1, 2
+
+EXPORTS = (
+    "spdy_plan_create", "spdy_plan_destroy", "spdy_plan_get_info", "spdy_plan_get_bands",
+    "spdy_workspace_bytes", "spdy_solve_batch", "spdy_solve_batch_host", "spdy_solve_batch_simple",
+    "spdy_plan_check_status", "spdy_plan_enable_timing", "spdy_plan_last_timing", "spdy_strerror", "spdy_last_cuda_error", "spdy_version",
+)
+
+
+class SpdyOptions(ctypes.Structure):
+    _fields_ = [("table_format", ctypes.c_int32), ("threads", ctypes.c_int32),
+                ("cluster", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
+
+
+class SpdyPlanInfo(ctypes.Structure):
+    _fields_ = [("L", ctypes.c_int32), ("K", ctypes.c_int32), ("B", ctypes.c_int32),
+                ("feasible", ctypes.c_int32), ("max_width", ctypes.c_int32),
+                ("span", ctypes.c_int32), ("threads", ctypes.c_int32), ("cluster", ctypes.c_int32),
+                ("table_format", ctypes.c_int32), ("ctas_per_sm", ctypes.c_int32),
+                ("sm_count", ctypes.c_int32), ("reserved0", ctypes.c_int32),
+                ("smem_bytes", ctypes.c_int64), ("table_bytes_per_candidate", ctypes.c_int64),
+                ("band_cells", ctypes.c_int64), ("useful_updates", ctypes.c_int64),
+                ("issued_updates", ctypes.c_int64), ("nominal_updates", ctypes.c_int64)]
+
+    def as_dict(self) -> dict:
+        return {name: int(getattr(self, name)) for name, _ in self._fields_ if name != "reserved0"}
+
+
+class SpdyError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        lib = _load()
+        text = lib.spdy_strerror(status).decode()
+        extra = f" (cudaError {lib.spdy_last_cuda_error()})" if status == -4 else ""
+        super().__init__(f"{where}: {text}{extra} [{status}]")
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                           "`python -m paper_2201_13096_b200.build` (needs nvcc); "
+                           "there is no fallback implementation")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    lib.spdy_plan_create.restype = ctypes.c_int
+    lib.spdy_plan_create.argtypes = [ctypes.POINTER(vp), vp, i32, i32, i32, ctypes.c_int,
+                                     ctypes.POINTER(SpdyOptions)]
+    lib.spdy_plan_destroy.restype = None
+    lib.spdy_plan_destroy.argtypes = [vp]
+    lib.spdy_plan_get_info.restype = ctypes.c_int
+    lib.spdy_plan_get_info.argtypes = [vp, ctypes.POINTER(SpdyPlanInfo)]
+    lib.spdy_plan_get_bands.restype = ctypes.c_int
+    lib.spdy_plan_get_bands.argtypes = [vp, vp, vp]
+    lib.spdy_workspace_bytes.restype = ctypes.c_size_t
+    lib.spdy_workspace_bytes.argtypes = [vp, i64]
+    lib.spdy_solve_batch.restype = ctypes.c_int
+    lib.spdy_solve_batch.argtypes = [vp, vp, i64, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.spdy_solve_batch_host.restype = ctypes.c_int
+    lib.spdy_solve_batch_host.argtypes = [vp, vp, i64, vp, vp, vp, vp]
+    lib.spdy_solve_batch_simple.restype = ctypes.c_int
+    lib.spdy_solve_batch_simple.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
+    lib.spdy_plan_check_status.restype = ctypes.c_int
+    lib.spdy_plan_check_status.argtypes = [vp, vp]
+    lib.spdy_plan_enable_timing.restype = ctypes.c_int
+    lib.spdy_plan_enable_timing.argtypes = [vp, ctypes.c_int]
+    lib.spdy_plan_last_timing.restype = ctypes.c_int
+    lib.spdy_plan_last_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
+                                          ctypes.POINTER(ctypes.c_float)]
+    lib.spdy_strerror.restype = ctypes.c_char_p
+    lib.spdy_strerror.argtypes = [ctypes.c_int]
+    lib.spdy_last_cuda_error.restype = ctypes.c_int
+    lib.spdy_version.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def library():
+    """The loaded ``ctypes.CDLL`` (raises if the library has not been built)."""
+    return _load()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise SpdyError(status, where)
+
+
+def _stream_handle(stream) -> Optional[int]:
+    import torch
+
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class Plan:
+    """``spdy_plan``: everything that depends only on ``times`` and ``B``."""
+
+    def __init__(self, times, B: int, device: int = 0, table_format: int = SPDY_TABLE_DEFAULT,
+                 threads: int = 0, cluster: int = 0):
+        lib = _load()
+        t = np.ascontiguousarray(np.asarray(times), dtype=np.int32)
+        if t.ndim != 2:
+            raise ValueError("times must be [L][K]")
+        self.L, self.K, self.B, self.device = int(t.shape[0]), int(t.shape[1]), int(B), int(device)
+        opts = SpdyOptions(table_format=table_format, threads=threads, cluster=cluster)
+        handle = ctypes.c_void_p()
+        _check(lib.spdy_plan_create(ctypes.byref(handle), t.ctypes.data_as(ctypes.c_void_p),
+                                    self.L, self.K, self.B, self.device, ctypes.byref(opts)),
+               "spdy_plan_create")
+        self._h = handle
+        self._ws = None
+
+    def close(self):
+        if getattr(self, "_h", None):
+            _load().spdy_plan_destroy(self._h)
+            self._h = None
+        self._ws = None
+
+    __del__ = close
+
+    @property
+    def info(self) -> dict:
+        out = SpdyPlanInfo()
+        _check(_load().spdy_plan_get_info(self._h, ctypes.byref(out)), "spdy_plan_get_info")
+        return out.as_dict()
+
+    def bands(self):
+        lo = np.empty(self.L, np.int32)
+        width = np.empty(self.L, np.int32)
+        _check(_load().spdy_plan_get_bands(self._h, lo.ctypes.data_as(ctypes.c_void_p),
+                                           width.ctypes.data_as(ctypes.c_void_p)),
+               "spdy_plan_get_bands")
+        return lo, width
+
+    def workspace_bytes(self, N: int) -> int:
+        return int(_load().spdy_workspace_bytes(self._h, int(N)))
+
+    def enable_timing(self, on: bool = True):
+        _check(_load().spdy_plan_enable_timing(self._h, int(on)), "spdy_plan_enable_timing")
+
+    def last_timing(self):
+        """(forward_ms, walkback_ms) of the last solve; waits for it."""
+        f, w = ctypes.c_float(), ctypes.c_float()
+        _check(_load().spdy_plan_last_timing(self._h, ctypes.byref(f), ctypes.byref(w)),
+               "spdy_plan_last_timing")
+        return float(f.value), float(w.value)
+
+    def check_status(self, stream=None):
+        _check(_load().spdy_plan_check_status(self._h, _stream_handle(stream)),
+               "spdy_plan_check_status")
+
+
+def solve_batch(plan: Plan, errors, profile=None, cost=None, time_used=None, workspace=None,
+                stream=None):
+    """``spdy_solve_batch`` on device tensors.  ``errors`` is a contiguous CUDA fp32 tensor
+    [N][L][K]; outputs and workspace are allocated with torch when not given.  Asynchronous on
+    ``stream`` (default: torch's current stream).  Returns (profile u8 [N][L], cost f32 [N],
+    time_used i32 [N])."""
+    import torch
+
+    if not (errors.is_cuda and errors.dtype == torch.float32 and errors.is_contiguous()):
+        raise ValueError("errors must be a contiguous CUDA float32 tensor")
+    if errors.dim() != 3 or errors.shape[1] != plan.L or errors.shape[2] != plan.K:
+        raise ValueError("errors must be [N][L][K] matching the plan")
+    N = int(errors.shape[0])
+    dev = errors.device
+    if profile is None:
+        profile = torch.empty((N, plan.L), dtype=torch.uint8, device=dev)
+    if cost is None:
+        cost = torch.empty(N, dtype=torch.float32, device=dev)
+    if time_used is None:
+        time_used = torch.empty(N, dtype=torch.int32, device=dev)
+    if workspace is None:
+        need = plan.workspace_bytes(N)
+        if plan._ws is None or plan._ws.numel() < need or plan._ws.device != dev:
+            plan._ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        workspace = plan._ws
+    _check(_load().spdy_solve_batch(plan._h, errors.data_ptr(), N, profile.data_ptr(),
+                                    cost.data_ptr(), time_used.data_ptr(), workspace.data_ptr(),
+                                    workspace.numel() * workspace.element_size(),
+                                    _stream_handle(stream)), "spdy_solve_batch")
+    return profile, cost, time_used
+
+
+def solve_batch_host(plan: Plan, errors: np.ndarray, profile=None, cost=None, time_used=None,
+                     stream=None):
+    """``spdy_solve_batch_host``: NumPy (or pinned torch CPU) buffers in and out, copies included."""
+    def addr(x):
+        return x.ctypes.data if isinstance(x, np.ndarray) else x.data_ptr()
+
+    N = int(errors.shape[0])
+    if profile is None:
+        profile = np.empty((N, plan.L), np.uint8)
+    if cost is None:
+        cost = np.empty(N, np.float32)
+    if time_used is None:
+        time_used = np.empty(N, np.int32)
+    _check(_load().spdy_solve_batch_host(plan._h, addr(errors), N, addr(profile), addr(cost),
+                                         addr(time_used), _stream_handle(stream)),
+           "spdy_solve_batch_host")
+    return profile, cost, time_used
+
+
+def solve_batch_simple(errors, times, B: int, stream=None):
+    """``spdy_solve_batch_simple``: the one-shot call (errors, times on the device, budget) ->
+    (profile, cost, time_used); synchronous."""
+    import torch
+
+    N, L, K = (int(x) for x in errors.shape)
+    dev = errors.device
+    profile = torch.empty((N, L), dtype=torch.uint8, device=dev)
+    cost = torch.empty(N, dtype=torch.float32, device=dev)
+    time_used = torch.empty(N, dtype=torch.int32, device=dev)
+    _check(_load().spdy_solve_batch_simple(errors.data_ptr(), times.data_ptr(), N, L, K, int(B),
+                                           profile.data_ptr(), cost.data_ptr(),
+                                           time_used.data_ptr(), _stream_handle(stream)),
+           "spdy_solve_batch_simple")
+    return profile, cost, time_used

@@ -1,0 +1,984 @@
+// Batched SPDY dynamic program for B200 (sm_100a): host plan, kernels and the C ABI.
+//
+// One candidate = one min-plus dynamic program over L layers (Section 3.2, Eq. 2-3) followed by
+// the final minimum over the budget axis and the walk back through the choice table (Appendix A,
+// Algorithm 1).  The forward kernel keeps two band-limited DP rows in shared memory and streams
+// one table row per layer to global memory; a second kernel walks the table back.
+//
+// Bit-exactness contract: every cell value is produced by exactly one fp32 round-to-nearest add
+// (previous-row value + error) and compared with strict "<" in ascending choice order, so the
+// results equal a plain sequential evaluation of Algorithm 1 with Eq. 2's bucket range.
+#include "../../include/spdy_dp.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+#define SPDY_CUDA_TRY(expr)                                  \
+    do {                                                     \
+        cudaError_t err__ = (expr);                          \
+        if (err__ != cudaSuccess) {                          \
+            g_last_cuda_error = static_cast<int>(err__);     \
+            return SPDY_ERR_CUDA;                            \
+        }                                                    \
+    } while (0)
+
+// ----------------------------------------------------------------------------------------------
+// Device-side layout
+// ----------------------------------------------------------------------------------------------
+
+// Row l (1-based; stored at index l-1) lives on the band [lo, lo + width).  A band cell is
+// addressed by t_rel = t - lo.  `rowoff` is where the row starts inside one candidate's table,
+// in cells, always a multiple of the span.
+struct LayerDesc {
+    int32_t width;
+    uint32_t rowoff;
+    int32_t lo;
+    int32_t mn;  // smallest usable time of the layer: lo_l = lo_{l-1} + mn
+};
+
+// One (layer, choice) pair in band coordinates: the choice contributes to cells t_rel in [a, b]
+// and reads the previous row at t_rel - a.  An unusable choice has b < a.
+struct TapRange {
+    int32_t a;
+    int32_t b;
+};
+
+struct FwdArgs {
+    const float *errors;      // [N][L][K]
+    const TapRange *taps;     // [L][K]
+    const LayerDesc *layers;  // [L]
+    void *table;              // wave-local walk-back table
+    float *cost;              // [N]
+    int32_t *time_used;       // [N]
+    int64_t pitch;            // table cells per candidate
+    int64_t n_first;          // first candidate of this wave
+    int32_t L, K;
+    int32_t row_stride;       // floats per shared-memory row buffer
+};
+
+__device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
+
+// Cells a warp owns in one pass: SPAN = 32*R consecutive band cells, lane i taking cells
+// i, i+32, ... so that every shared-memory access is lane-consecutive (conflict-free) whatever
+// the shift.  Both row buffers carry SPAN cells of +inf on either side of the band: a warp whose
+// span only partly overlaps a choice's range then reads +inf for the cells outside it, and no
+// per-cell bounds check is needed.
+//
+// Table layouts (internal, only the walk-back kernel reads them):
+//   ARG:  one byte per cell; inside a span the byte of cell u = 32*j + lane sits at lane*R + j,
+//         so each lane writes its R bytes with 16-byte stores.
+//   !ARG: one float per cell in natural order.
+template <int R, bool ARG, int NT, int MINB>
+__global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs args)
+{
+    constexpr int SPAN = 32 * R;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *rows = reinterpret_cast<float *>(smem_raw);
+    int4 *tap_buf = reinterpret_cast<int4 *>(rows + 2 * static_cast<size_t>(args.row_stride));
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    constexpr int NWARPS = NT / 32;
+    const int L = args.L, K = args.K;
+    const int64_t n_local = blockIdx.x;
+    const int64_t n = args.n_first + n_local;
+    const float *err_n = args.errors + n * L * K;
+    const float INF = pos_inf();
+
+    // Both buffers start as +inf everywhere; D_0 is +0 at t = 0 (Eq. 3 via a virtual row 0).
+    for (int i = tid; i < 2 * args.row_stride; i += NT) rows[i] = INF;
+    if (tid < K) {
+        const TapRange tr = args.taps[tid];
+        tap_buf[tid] = make_int4(tr.a, tr.b, __float_as_int(err_n[tid]), 0);
+    }
+    __syncthreads();
+    if (tid == 0) rows[SPAN] = 0.0f;
+    __syncthreads();
+
+    for (int l = 0; l < L; ++l) {
+        const float *prev = rows + (l & 1) * args.row_stride + SPAN;
+        float *cur = rows + ((l + 1) & 1) * args.row_stride + SPAN;
+        const int4 *taps = tap_buf + (l & 1) * K;
+        const LayerDesc ld = args.layers[l];
+        const int nspans = (ld.width + SPAN - 1) / SPAN;
+
+        // Fetch the next layer's choices early; they are parked in shared memory after the pass.
+        int4 next_tap = make_int4(0, -1, 0, 0);
+        const bool have_next = (l + 1 < L) && (tid < K);
+        if (have_next) {
+            const TapRange tr = args.taps[(l + 1) * K + tid];
+            next_tap = make_int4(tr.a, tr.b, __float_as_int(err_n[(l + 1) * K + tid]), 0);
+        }
+
+        for (int span = warp; span < nspans; span += NWARPS) {
+            const int s = span * SPAN;
+            float best[R];
+            int idx[R];
+#pragma unroll
+            for (int j = 0; j < R; ++j) {
+                best[j] = INF;
+                idx[j] = 0xFF;
+            }
+            const float *prev_lane = prev + s + lane;
+#pragma unroll 1
+            for (int k = 0; k < K; ++k) {
+                const int4 tp = taps[k];
+                if (s + SPAN > tp.x && s <= tp.y) {  // warp-uniform
+                    const float *src = prev_lane - tp.x;
+                    const float e = __int_as_float(tp.z);
+#pragma unroll
+                    for (int j = 0; j < R; ++j) {
+                        const float v = __fadd_rn(src[j * 32], e);
+                        if (ARG) {
+                            const bool better = v < best[j];
+                            best[j] = better ? v : best[j];
+                            idx[j] = better ? k : idx[j];
+                        } else {
+                            best[j] = fminf(best[j], v);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < R; ++j) cur[s + j * 32 + lane] = best[j];
+            if (ARG) {
+                unsigned char *P = static_cast<unsigned char *>(args.table) +
+                                   (n_local * args.pitch + ld.rowoff + s);
+                if (R % 16 == 0) {
+#pragma unroll
+                    for (int q = 0; q < R / 16; ++q) {
+                        uint4 w;
+                        w.x = idx[16 * q + 0] | (idx[16 * q + 1] << 8) | (idx[16 * q + 2] << 16) | (idx[16 * q + 3] << 24);
+                        w.y = idx[16 * q + 4] | (idx[16 * q + 5] << 8) | (idx[16 * q + 6] << 16) | (idx[16 * q + 7] << 24);
+                        w.z = idx[16 * q + 8] | (idx[16 * q + 9] << 8) | (idx[16 * q + 10] << 16) | (idx[16 * q + 11] << 24);
+                        w.w = idx[16 * q + 12] | (idx[16 * q + 13] << 8) | (idx[16 * q + 14] << 16) | (idx[16 * q + 15] << 24);
+                        reinterpret_cast<uint4 *>(P + lane * R)[q] = w;
+                    }
+                } else {
+                    static_assert(R % 16 == 0 || R == 8, "R must be 8 or a multiple of 16");
+                    uint2 w;
+                    w.x = idx[0] | (idx[1] << 8) | (idx[2] << 16) | (idx[3] << 24);
+                    w.y = idx[4] | (idx[5] << 8) | (idx[6] << 16) | (idx[7] << 24);
+                    *reinterpret_cast<uint2 *>(P + lane * R) = w;
+                }
+            } else {
+                float *D = static_cast<float *>(args.table) + (n_local * args.pitch + ld.rowoff + s) + lane;
+#pragma unroll
+                for (int j = 0; j < R; ++j) D[j * 32] = best[j];
+            }
+        }
+        // Cells [width, width + SPAN) of the new row must read as +inf for the next layer.  The
+        // spans above wrote +inf up to nspans*SPAN (their out-of-range cells saw only +inf
+        // sources); one more span of +inf covers the rest.
+        for (int i = tid; i < SPAN; i += NT) cur[nspans * SPAN + i] = INF;
+        if (have_next) tap_buf[((l + 1) & 1) * K + tid] = next_tap;
+        __syncthreads();
+    }
+
+    // min over t <= B of D_L[t], lowest t among equals (the band's upper end never exceeds B).
+    const float *last = rows + (L & 1) * args.row_stride + SPAN;
+    const LayerDesc ld = args.layers[L - 1];
+    float bv = INF;
+    int bt = 0x7fffffff;
+    for (int t = tid; t < ld.width; t += NT) {
+        const float v = last[t];
+        if (v < bv) {
+            bv = v;
+            bt = t;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+        const int ot = __shfl_xor_sync(0xffffffffu, bt, off);
+        if (ov < bv || (ov == bv && ot < bt)) {
+            bv = ov;
+            bt = ot;
+        }
+    }
+    __shared__ float red_v[32];
+    __shared__ int red_t[32];
+    if (lane == 0) {
+        red_v[warp] = bv;
+        red_t[warp] = bt;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        bv = lane < NWARPS ? red_v[lane] : INF;
+        bt = lane < NWARPS ? red_t[lane] : 0x7fffffff;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+            const int ot = __shfl_xor_sync(0xffffffffu, bt, off);
+            if (ov < bv || (ov == bv && ot < bt)) {
+                bv = ov;
+                bt = ot;
+            }
+        }
+        if (lane == 0) {
+            const bool feasible = bv < INF;
+            args.cost[n] = feasible ? bv : INF;
+            args.time_used[n] = feasible ? ld.lo + bt : -1;
+        }
+    }
+}
+
+struct BackArgs {
+    const float *errors;      // [N][L][K]
+    const int32_t *times;     // [L][K]
+    const LayerDesc *layers;  // [L]
+    const void *table;
+    const float *cost;
+    const int32_t *time_used;
+    uint8_t *profile;         // [N][L]
+    int32_t *status;          // device word, set non-zero if a self-check fails
+    int64_t pitch;
+    int64_t n_first;
+    int64_t n_count;
+    int32_t L, K, R;
+};
+
+// Walk back through the byte table (end of Algorithm 1): one thread per candidate.
+__global__ void spdy_backtrack_arg_kernel(const BackArgs args)
+{
+    const int64_t n_local = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    if (n_local >= args.n_count) return;
+    const int64_t n = args.n_first + n_local;
+    const int L = args.L, K = args.K, R = args.R;
+    const int span = 32 * R;
+    uint8_t *prof = args.profile + n * L;
+    int t = args.time_used[n];
+    if (t < 0) {
+        for (int l = 0; l < L; ++l) prof[l] = 0xFF;
+        return;
+    }
+    const unsigned char *P = static_cast<const unsigned char *>(args.table) + n_local * args.pitch;
+    bool ok = true;
+    for (int l = L - 1; l >= 0; --l) {
+        const LayerDesc ld = args.layers[l];
+        const int t_rel = t - ld.lo;
+        int k = 0xFF;
+        if (ok && t_rel >= 0 && t_rel < ld.width) {
+            const int u = t_rel % span;
+            k = P[ld.rowoff + (t_rel - u) + (u & 31) * R + (u >> 5)];
+        }
+        if (k >= K) {
+            ok = false;
+            k = 0xFF;
+        } else {
+            t -= args.times[l * K + k];
+        }
+        prof[l] = static_cast<uint8_t>(k);
+    }
+    if (!ok || t != 0) atomicExch(args.status, 1);
+}
+
+// Walk back through stored row values: one warp per candidate.  At (l, t) the winning choice is
+// the lowest k whose fp32 sum D_{l-1}[t - times[l][k]] + errors[n][l][k] equals D_l[t] bit for
+// bit; the forward pass formed D_l[t] as the minimum of exactly these sums.
+__global__ void spdy_backtrack_row_kernel(const BackArgs args)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t n_local = (blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x) >> 5;
+    if (n_local >= args.n_count) return;
+    const int64_t n = args.n_first + n_local;
+    const int L = args.L, K = args.K;
+    uint8_t *prof = args.profile + n * L;
+    int t = args.time_used[n];
+    if (t < 0) {
+        for (int l = lane; l < L; l += 32) prof[l] = 0xFF;
+        return;
+    }
+    const float INF = pos_inf();
+    const float *D = static_cast<const float *>(args.table) + n_local * args.pitch;
+    const float *err_n = args.errors + n * L * K;
+    float target = args.cost[n];
+    bool ok = true;
+    for (int l = L - 1; l >= 0; --l) {
+        const LayerDesc ld = args.layers[l];
+        const int t_rel = t - ld.lo;
+        int prev_width = 1;
+        uint32_t prev_off = 0;
+        if (l > 0) {
+            const LayerDesc pl = args.layers[l - 1];
+            prev_width = pl.width;
+            prev_off = pl.rowoff;
+        }
+        int found_k = 0xFF;
+        float found_prev = INF;
+        int found_tau = 0;
+        for (int k0 = 0; k0 < K && found_k == 0xFF; k0 += 32) {
+            const int k = k0 + lane;
+            float pv = INF;
+            int tau = 0;
+            bool match = false;
+            if (k < K) {
+                tau = args.times[l * K + k];
+                const int64_t src = static_cast<int64_t>(t_rel) - (static_cast<int64_t>(tau) - ld.mn);
+                if (src >= 0 && src < prev_width) {
+                    pv = (l == 0) ? 0.0f : D[prev_off + src];
+                    const float v = __fadd_rn(pv, err_n[l * K + k]);
+                    match = (v == target) && (pv < INF);
+                }
+            }
+            const unsigned ballot = __ballot_sync(0xffffffffu, match);
+            if (ballot) {
+                const int src_lane = __ffs(ballot) - 1;
+                found_k = k0 + src_lane;
+                found_prev = __shfl_sync(0xffffffffu, pv, src_lane);
+                found_tau = __shfl_sync(0xffffffffu, tau, src_lane);
+            }
+        }
+        if (found_k == 0xFF) {
+            ok = false;
+            if (lane == 0) prof[l] = 0xFF;
+        } else {
+            if (lane == 0) prof[l] = static_cast<uint8_t>(found_k);
+            t -= found_tau;
+            target = found_prev;
+        }
+        if (!ok) {
+            for (int ll = l - 1 - lane; ll >= 0; ll -= 32) prof[ll] = 0xFF;
+            break;
+        }
+    }
+    if ((!ok || t != 0) && lane == 0) atomicExch(args.status, 1);
+}
+
+__global__ void spdy_fill_infeasible_kernel(uint8_t *profile, float *cost, int32_t *time_used,
+                                            int64_t N, int32_t L)
+{
+    const int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    const int64_t total = N * L;
+    for (int64_t j = i; j < total; j += static_cast<int64_t>(gridDim.x) * blockDim.x) profile[j] = 0xFF;
+    if (i < N) {
+        cost[i] = pos_inf();
+        time_used[i] = -1;
+    }
+}
+
+// ----------------------------------------------------------------------------------------------
+// Kernel table
+// ----------------------------------------------------------------------------------------------
+
+using FwdKernel = void (*)(const FwdArgs);
+
+struct FwdVariant {
+    int R;
+    bool arg;
+    int threads;
+    FwdKernel fn;
+};
+
+#define SPDY_VARIANT(R, ARG, NT, MINB) \
+    FwdVariant { R, ARG, NT, spdy_forward_kernel<R, ARG, NT, MINB> }
+
+const FwdVariant kVariants[] = {
+    SPDY_VARIANT(16, true, 128, 4),  SPDY_VARIANT(16, true, 256, 3),
+    SPDY_VARIANT(16, true, 512, 1),  SPDY_VARIANT(16, true, 1024, 1),
+    SPDY_VARIANT(16, false, 128, 4), SPDY_VARIANT(16, false, 256, 3),
+    SPDY_VARIANT(16, false, 512, 1), SPDY_VARIANT(16, false, 1024, 1),
+    SPDY_VARIANT(8, true, 128, 4),   SPDY_VARIANT(8, true, 256, 4),
+    SPDY_VARIANT(8, true, 512, 2),   SPDY_VARIANT(8, true, 1024, 1),
+    SPDY_VARIANT(8, false, 128, 4),  SPDY_VARIANT(8, false, 256, 4),
+    SPDY_VARIANT(8, false, 512, 2),  SPDY_VARIANT(8, false, 1024, 1),
+};
+
+const FwdVariant *find_variant(int R, bool arg, int threads)
+{
+    for (const FwdVariant &v : kVariants)
+        if (v.R == R && v.arg == arg && v.threads == threads) return &v;
+    return nullptr;
+}
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+}  // namespace
+
+// ----------------------------------------------------------------------------------------------
+// Plan
+// ----------------------------------------------------------------------------------------------
+
+struct spdy_plan {
+    int32_t L = 0, K = 0, B = 0;
+    int device = -1;
+    bool feasible = false;
+    int R = 16;
+    int threads = 256;
+    int cluster = 1;
+    int table_format = SPDY_TABLE_ARG_U8;
+    int ctas_per_sm = 0;
+    int sm_count = 148;
+    int64_t smem_bytes = 0;
+    int32_t row_stride = 0;
+    int64_t pitch = 0;  // table cells per candidate
+    int64_t band_cells = 0, useful_updates = 0, issued_updates = 0;
+    int32_t max_width = 0;
+    std::vector<int32_t> times;
+    std::vector<LayerDesc> layers;
+    std::vector<TapRange> taps;
+    const FwdVariant *variant = nullptr;
+    // device tables (one allocation)
+    unsigned char *d_blob = nullptr;
+    int32_t *d_times = nullptr;
+    LayerDesc *d_layers = nullptr;
+    TapRange *d_taps = nullptr;
+    int32_t *d_status = nullptr;
+    // optional event timing of the last solve (three events per wave)
+    bool timing = false;
+    std::vector<cudaEvent_t> events;
+    size_t events_used = 0;
+    // staging for the host-buffer entry point
+    unsigned char *d_arena = nullptr;
+    size_t arena_bytes = 0;
+};
+
+namespace {
+
+int64_t cell_bytes(const spdy_plan *p) { return p->table_format == SPDY_TABLE_ROW_F32 ? 4 : 1; }
+
+// Live band of every row and the range of every (layer, choice) pair.
+//   lo_l = sum_{j<=l} mn_j,  hi_l = min(B, sum_{j<=l} mx_j, B - sum_{j>l} mn_j)
+// with mn/mx the smallest/largest usable (<= B) time of a layer.  A cell below lo_l is
+// unreachable, a cell above hi_l is unreachable or cannot be completed within B; a cell inside
+// the band depends only on cells inside the previous band.
+int build_bands(spdy_plan *p)
+{
+    const int L = p->L, K = p->K;
+    const int64_t B = p->B;
+    std::vector<int64_t> mn(L), mx(L);
+    p->feasible = true;
+    for (int l = 0; l < L; ++l) {
+        int64_t lo = -1, hi = -1;
+        for (int k = 0; k < K; ++k) {
+            const int64_t tau = p->times[static_cast<size_t>(l) * K + k];
+            if (tau < 0) return SPDY_ERR_INVALID_ARG;
+            if (tau > B) continue;
+            lo = (lo < 0 || tau < lo) ? tau : lo;
+            hi = tau > hi ? tau : hi;
+        }
+        if (lo < 0) p->feasible = false;
+        mn[l] = lo < 0 ? 0 : lo;
+        mx[l] = hi < 0 ? 0 : hi;
+    }
+    int64_t total_mn = 0;
+    for (int l = 0; l < L; ++l) total_mn += mn[l];
+    if (total_mn > B) p->feasible = false;
+
+    p->layers.assign(L, LayerDesc{0, 0, 0, 0});
+    p->taps.assign(static_cast<size_t>(L) * K, TapRange{0, -1});
+    p->band_cells = p->useful_updates = 0;
+    p->max_width = 0;
+    if (!p->feasible) return SPDY_OK;
+
+    int64_t sum_mn = 0, sum_mx = 0, prev_width = 1;
+    for (int l = 0; l < L; ++l) {
+        sum_mn += mn[l];
+        sum_mx += mx[l];
+        const int64_t lo = sum_mn;
+        const int64_t hi = std::min<int64_t>(std::min<int64_t>(B, sum_mx), B - (total_mn - sum_mn));
+        const int64_t width = hi - lo + 1;
+        p->layers[l].width = static_cast<int32_t>(width);
+        p->layers[l].lo = static_cast<int32_t>(lo);
+        p->layers[l].mn = static_cast<int32_t>(mn[l]);
+        p->band_cells += width;
+        p->max_width = std::max<int32_t>(p->max_width, static_cast<int32_t>(width));
+        for (int k = 0; k < K; ++k) {
+            const int64_t tau = p->times[static_cast<size_t>(l) * K + k];
+            if (tau > B) continue;
+            const int64_t a = tau - mn[l];
+            const int64_t b = std::min<int64_t>(width - 1, prev_width - 1 + a);
+            if (b < a) continue;
+            p->taps[static_cast<size_t>(l) * K + k] = TapRange{static_cast<int32_t>(a), static_cast<int32_t>(b)};
+            p->useful_updates += b - a + 1;
+        }
+        prev_width = width;
+    }
+    return SPDY_OK;
+}
+
+// Row offsets, table pitch and issued work for a given span.
+int layout_table(spdy_plan *p)
+{
+    const int span = 32 * p->R;
+    int64_t off = 0;
+    p->issued_updates = 0;
+    for (int l = 0; l < p->L; ++l) {
+        if (off > 0xffffffffLL) return SPDY_ERR_UNSUPPORTED;
+        p->layers[l].rowoff = static_cast<uint32_t>(off);
+        const int64_t nspans = (p->layers[l].width + span - 1) / span;
+        off += nspans * span;
+        for (int k = 0; k < p->K; ++k) {
+            const TapRange tr = p->taps[static_cast<size_t>(l) * p->K + k];
+            if (tr.b < tr.a) continue;
+            const int64_t s_first = tr.a / span;  // first span whose end lies above a
+            const int64_t s_last = std::min<int64_t>(nspans - 1, tr.b / span);
+            if (s_last >= s_first) p->issued_updates += (s_last - s_first + 1) * span;
+        }
+    }
+    p->pitch = off;
+    p->row_stride = static_cast<int32_t>(round_up(p->max_width, span) + 2 * span);
+    p->smem_bytes = 2LL * p->row_stride * 4 + 2LL * p->K * 16;
+    return SPDY_OK;
+}
+
+int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
+{
+    int64_t smem_per_sm = 233472, smem_per_block = 232448;
+    p->sm_count = 148;
+    if (p->device >= 0) {
+        int v = 0;
+        SPDY_CUDA_TRY(cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerMultiprocessor, p->device));
+        smem_per_sm = v;
+        SPDY_CUDA_TRY(cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device));
+        smem_per_block = v;
+        SPDY_CUDA_TRY(cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, p->device));
+        p->sm_count = v;
+    }
+    p->table_format = (opts && opts->table_format) ? opts->table_format : SPDY_TABLE_ARG_U8;
+    if (p->table_format != SPDY_TABLE_ARG_U8 && p->table_format != SPDY_TABLE_ROW_F32)
+        return SPDY_ERR_INVALID_ARG;
+    p->cluster = (opts && opts->cluster) ? opts->cluster : 1;
+    if (p->cluster != 1) return SPDY_ERR_UNSUPPORTED;
+
+    p->R = 16;
+    int rc = layout_table(p);
+    if (rc != SPDY_OK) return rc;
+    if (p->smem_bytes > smem_per_block) {
+        p->R = 8;  // narrower guard bands
+        rc = layout_table(p);
+        if (rc != SPDY_OK) return rc;
+        if (p->smem_bytes > smem_per_block) return SPDY_ERR_UNSUPPORTED;
+    }
+    const int64_t by_smem = std::max<int64_t>(1, smem_per_sm / (p->smem_bytes + 1024));
+    int threads;
+    if (opts && opts->threads) {
+        threads = opts->threads;
+    } else if (by_smem >= 8) {
+        threads = 128;
+    } else if (by_smem >= 3) {
+        threads = 256;
+    } else if (by_smem == 2) {
+        threads = 512;
+    } else {
+        threads = 1024;
+    }
+    if (!(opts && opts->threads) && threads < p->K) threads = 256;  // one thread per choice stages the next layer
+    if (threads < p->K) return SPDY_ERR_INVALID_ARG;
+    p->threads = threads;
+    p->variant = find_variant(p->R, p->table_format == SPDY_TABLE_ARG_U8, threads);
+    if (!p->variant) return SPDY_ERR_INVALID_ARG;
+    p->ctas_per_sm = static_cast<int>(std::min<int64_t>(by_smem, 2048 / threads));
+    if (p->device >= 0) {
+        SPDY_CUDA_TRY(cudaFuncSetAttribute(p->variant->fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           static_cast<int>(p->smem_bytes)));
+        int occ = 0;
+        SPDY_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, p->variant->fn, threads,
+                                                                    static_cast<size_t>(p->smem_bytes)));
+        if (occ < 1) return SPDY_ERR_UNSUPPORTED;
+        p->ctas_per_sm = occ;
+    }
+    return SPDY_OK;
+}
+
+int upload_tables(spdy_plan *p)
+{
+    const size_t n_times = static_cast<size_t>(p->L) * p->K;
+    const size_t off_layers = round_up(n_times * sizeof(int32_t), 256);
+    const size_t off_taps = off_layers + round_up(p->L * sizeof(LayerDesc), 256);
+    const size_t off_status = off_taps + round_up(n_times * sizeof(TapRange), 256);
+    const size_t total = off_status + 256;
+    std::vector<unsigned char> host(total, 0);
+    std::memcpy(host.data(), p->times.data(), n_times * sizeof(int32_t));
+    std::memcpy(host.data() + off_layers, p->layers.data(), p->L * sizeof(LayerDesc));
+    std::memcpy(host.data() + off_taps, p->taps.data(), n_times * sizeof(TapRange));
+    cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&p->d_blob), total);
+    if (err != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(err);
+        p->d_blob = nullptr;
+        return err == cudaErrorMemoryAllocation ? SPDY_ERR_NO_MEMORY : SPDY_ERR_CUDA;
+    }
+    SPDY_CUDA_TRY(cudaMemcpy(p->d_blob, host.data(), total, cudaMemcpyHostToDevice));
+    p->d_times = reinterpret_cast<int32_t *>(p->d_blob);
+    p->d_layers = reinterpret_cast<LayerDesc *>(p->d_blob + off_layers);
+    p->d_taps = reinterpret_cast<TapRange *>(p->d_blob + off_taps);
+    p->d_status = reinterpret_cast<int32_t *>(p->d_blob + off_status);
+    return SPDY_OK;
+}
+
+struct DeviceGuard {
+    int saved = -1;
+    bool active = false;
+    int enter(int device)
+    {
+        SPDY_CUDA_TRY(cudaGetDevice(&saved));
+        if (saved != device) {
+            SPDY_CUDA_TRY(cudaSetDevice(device));
+            active = true;
+        }
+        return SPDY_OK;
+    }
+    ~DeviceGuard()
+    {
+        if (active) cudaSetDevice(saved);
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+int spdy_version(void) { return 1000; }
+
+int spdy_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char *spdy_strerror(int status)
+{
+    switch (status) {
+        case SPDY_OK: return "success";
+        case SPDY_ERR_INVALID_ARG: return "invalid argument";
+        case SPDY_ERR_WORKSPACE_TOO_SMALL: return "workspace too small for one candidate";
+        case SPDY_ERR_UNSUPPORTED: return "problem shape not supported on this device";
+        case SPDY_ERR_CUDA: return "CUDA runtime call failed";
+        case SPDY_ERR_NO_MEMORY: return "out of memory";
+        case SPDY_ERR_INTERNAL: return "internal self-check failed";
+        default: return "unknown status";
+    }
+}
+
+int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int32_t K, int32_t B,
+                     int device, const spdy_options *opts)
+{
+    if (!out) return SPDY_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!times_host || L < 1 || K < 1 || K > 255 || B < 0 || device < -1) return SPDY_ERR_INVALID_ARG;
+    if (opts) {
+        for (int i = 0; i < 5; ++i)
+            if (opts->reserved[i] != 0) return SPDY_ERR_INVALID_ARG;
+        if (opts->threads != 0 && (opts->threads % 32 != 0 || opts->threads < 64 || opts->threads > 1024))
+            return SPDY_ERR_INVALID_ARG;
+    }
+    spdy_plan *p = new (std::nothrow) spdy_plan();
+    if (!p) return SPDY_ERR_NO_MEMORY;
+    p->L = L;
+    p->K = K;
+    p->B = B;
+    p->device = device;
+    int rc = SPDY_OK;
+    try {
+        p->times.assign(times_host, times_host + static_cast<size_t>(L) * K);
+        rc = build_bands(p);
+        DeviceGuard guard;
+        if (rc == SPDY_OK && device >= 0) rc = guard.enter(device);
+        if (rc == SPDY_OK) rc = choose_launch_shape(p, opts);
+        if (rc == SPDY_OK && device >= 0) rc = upload_tables(p);
+    } catch (const std::bad_alloc &) {
+        rc = SPDY_ERR_NO_MEMORY;
+    }
+    if (rc != SPDY_OK) {
+        spdy_plan_destroy(p);
+        return rc;
+    }
+    *out = p;
+    return SPDY_OK;
+}
+
+void spdy_plan_destroy(spdy_plan *plan)
+{
+    if (!plan) return;
+    if (plan->d_blob || plan->d_arena) {
+        DeviceGuard guard;
+        guard.enter(plan->device);
+        if (plan->d_blob) cudaFree(plan->d_blob);
+        if (plan->d_arena) cudaFree(plan->d_arena);
+        for (cudaEvent_t e : plan->events) cudaEventDestroy(e);
+    }
+    delete plan;
+}
+
+int spdy_plan_get_info(const spdy_plan *plan, spdy_plan_info *info)
+{
+    if (!plan || !info) return SPDY_ERR_INVALID_ARG;
+    std::memset(info, 0, sizeof(*info));
+    info->L = plan->L;
+    info->K = plan->K;
+    info->B = plan->B;
+    info->feasible = plan->feasible ? 1 : 0;
+    info->max_width = plan->max_width;
+    info->span = 32 * plan->R;
+    info->threads = plan->threads;
+    info->cluster = plan->cluster;
+    info->table_format = plan->table_format;
+    info->ctas_per_sm = plan->ctas_per_sm;
+    info->sm_count = plan->sm_count;
+    info->smem_bytes = plan->smem_bytes;
+    info->table_bytes_per_candidate = plan->pitch * cell_bytes(plan);
+    info->band_cells = plan->band_cells;
+    info->useful_updates = plan->useful_updates;
+    info->issued_updates = plan->issued_updates;
+    info->nominal_updates = static_cast<int64_t>(plan->L) * plan->K * plan->B;
+    return SPDY_OK;
+}
+
+int spdy_plan_get_bands(const spdy_plan *plan, int32_t *lo_host, int32_t *width_host)
+{
+    if (!plan) return SPDY_ERR_INVALID_ARG;
+    for (int l = 0; l < plan->L; ++l) {
+        if (lo_host) lo_host[l] = plan->layers[l].lo;
+        if (width_host) width_host[l] = plan->layers[l].width;
+    }
+    return SPDY_OK;
+}
+
+size_t spdy_workspace_bytes(const spdy_plan *plan, int64_t N)
+{
+    if (!plan || N <= 0) return 0;
+    const int64_t per = std::max<int64_t>(256, round_up(plan->pitch * cell_bytes(plan), 256));
+    return static_cast<size_t>(per) * static_cast<size_t>(N);
+}
+
+int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
+                     uint8_t *profile_dev, float *cost_dev, int32_t *time_used_dev,
+                     void *workspace_dev, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!plan || plan->device < 0 || N < 0) return SPDY_ERR_INVALID_ARG;
+    if (N == 0) return SPDY_OK;
+    if (!errors_dev || !profile_dev || !cost_dev || !time_used_dev) return SPDY_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(errors_dev) % 4 != 0) return SPDY_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard;
+    int rc = guard.enter(plan->device);
+    if (rc != SPDY_OK) return rc;
+
+    if (!plan->feasible) {
+        const int blocks = static_cast<int>(std::min<int64_t>((N + 255) / 256, 65535));
+        spdy_fill_infeasible_kernel<<<blocks, 256, 0, stream>>>(profile_dev, cost_dev, time_used_dev, N, plan->L);
+        SPDY_CUDA_TRY(cudaGetLastError());
+        return SPDY_OK;
+    }
+    if (!workspace_dev || reinterpret_cast<uintptr_t>(workspace_dev) % 256 != 0) return SPDY_ERR_INVALID_ARG;
+    const size_t per = spdy_workspace_bytes(plan, 1);
+    const int64_t wave = static_cast<int64_t>(std::min<size_t>(workspace_bytes / per, static_cast<size_t>(N)));
+    if (wave < 1) return SPDY_ERR_WORKSPACE_TOO_SMALL;
+    // The table pitch handed to the kernels is in cells; `per` bytes per candidate keeps every
+    // candidate's table 256-byte aligned.
+    const int64_t pitch_cells = static_cast<int64_t>(per) / cell_bytes(plan);
+
+    spdy_plan *mplan = const_cast<spdy_plan *>(plan);  // timing state only
+    if (plan->timing) mplan->events_used = 0;
+    for (int64_t first = 0; first < N; first += wave) {
+        const int64_t count = std::min<int64_t>(wave, N - first);
+        cudaEvent_t *ev = nullptr;
+        if (plan->timing) {
+            while (mplan->events.size() < mplan->events_used + 3) {
+                cudaEvent_t e;
+                SPDY_CUDA_TRY(cudaEventCreate(&e));
+                mplan->events.push_back(e);
+            }
+            ev = &mplan->events[mplan->events_used];
+            mplan->events_used += 3;
+            SPDY_CUDA_TRY(cudaEventRecord(ev[0], stream));
+        }
+        FwdArgs fa;
+        fa.errors = errors_dev;
+        fa.taps = plan->d_taps;
+        fa.layers = plan->d_layers;
+        fa.table = workspace_dev;
+        fa.cost = cost_dev;
+        fa.time_used = time_used_dev;
+        fa.pitch = pitch_cells;
+        fa.n_first = first;
+        fa.L = plan->L;
+        fa.K = plan->K;
+        fa.row_stride = plan->row_stride;
+        // Grid x is limited to 2^31-1 CTAs, far above any wave that fits in memory.
+        plan->variant->fn<<<static_cast<unsigned>(count), plan->threads, static_cast<size_t>(plan->smem_bytes), stream>>>(fa);
+        SPDY_CUDA_TRY(cudaGetLastError());
+        if (ev) SPDY_CUDA_TRY(cudaEventRecord(ev[1], stream));
+
+        BackArgs ba;
+        ba.errors = errors_dev;
+        ba.times = plan->d_times;
+        ba.layers = plan->d_layers;
+        ba.table = workspace_dev;
+        ba.cost = cost_dev;
+        ba.time_used = time_used_dev;
+        ba.profile = profile_dev;
+        ba.status = plan->d_status;
+        ba.pitch = pitch_cells;
+        ba.n_first = first;
+        ba.n_count = count;
+        ba.L = plan->L;
+        ba.K = plan->K;
+        ba.R = plan->R;
+        if (plan->table_format == SPDY_TABLE_ARG_U8) {
+            const int bt = 64;
+            spdy_backtrack_arg_kernel<<<static_cast<unsigned>((count + bt - 1) / bt), bt, 0, stream>>>(ba);
+        } else {
+            const int bt = 128;  // 4 warps = 4 candidates per CTA
+            spdy_backtrack_row_kernel<<<static_cast<unsigned>((count * 32 + bt - 1) / bt), bt, 0, stream>>>(ba);
+        }
+        SPDY_CUDA_TRY(cudaGetLastError());
+        if (ev) SPDY_CUDA_TRY(cudaEventRecord(ev[2], stream));
+    }
+    return SPDY_OK;
+}
+
+int spdy_plan_enable_timing(spdy_plan *plan, int on)
+{
+    if (!plan || plan->device < 0) return SPDY_ERR_INVALID_ARG;
+    plan->timing = on != 0;
+    plan->events_used = 0;
+    return SPDY_OK;
+}
+
+int spdy_plan_last_timing(spdy_plan *plan, float *forward_ms_host, float *walkback_ms_host)
+{
+    if (!plan || plan->device < 0 || !plan->timing) return SPDY_ERR_INVALID_ARG;
+    DeviceGuard guard;
+    int rc = guard.enter(plan->device);
+    if (rc != SPDY_OK) return rc;
+    float fwd = 0.f, back = 0.f;
+    for (size_t i = 0; i + 3 <= plan->events_used && i + 3 <= plan->events.size(); i += 3) {
+        SPDY_CUDA_TRY(cudaEventSynchronize(plan->events[i + 2]));
+        float a = 0.f, b = 0.f;
+        SPDY_CUDA_TRY(cudaEventElapsedTime(&a, plan->events[i], plan->events[i + 1]));
+        SPDY_CUDA_TRY(cudaEventElapsedTime(&b, plan->events[i + 1], plan->events[i + 2]));
+        fwd += a;
+        back += b;
+    }
+    if (forward_ms_host) *forward_ms_host = fwd;
+    if (walkback_ms_host) *walkback_ms_host = back;
+    return SPDY_OK;
+}
+
+int spdy_plan_check_status(spdy_plan *plan, void *cuda_stream)
+{
+    if (!plan || plan->device < 0) return SPDY_ERR_INVALID_ARG;
+    DeviceGuard guard;
+    int rc = guard.enter(plan->device);
+    if (rc != SPDY_OK) return rc;
+    int32_t word = 0;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    SPDY_CUDA_TRY(cudaMemcpyAsync(&word, plan->d_status, sizeof(word), cudaMemcpyDeviceToHost, stream));
+    SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (word != 0) {
+        SPDY_CUDA_TRY(cudaMemsetAsync(plan->d_status, 0, sizeof(word), stream));
+        SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
+        return SPDY_ERR_INTERNAL;
+    }
+    return SPDY_OK;
+}
+
+int spdy_solve_batch_host(spdy_plan *plan, const float *errors_host, int64_t N,
+                          uint8_t *profile_host, float *cost_host, int32_t *time_used_host,
+                          void *cuda_stream)
+{
+    if (!plan || plan->device < 0 || N < 0) return SPDY_ERR_INVALID_ARG;
+    if (N == 0) return SPDY_OK;
+    if (!errors_host || !profile_host || !cost_host || !time_used_host) return SPDY_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard;
+    int rc = guard.enter(plan->device);
+    if (rc != SPDY_OK) return rc;
+
+    const size_t err_bytes = static_cast<size_t>(N) * plan->L * plan->K * sizeof(float);
+    const size_t off_profile = round_up(err_bytes, 256);
+    const size_t off_cost = off_profile + round_up(static_cast<size_t>(N) * plan->L, 256);
+    const size_t off_time = off_cost + round_up(static_cast<size_t>(N) * 4, 256);
+    const size_t off_ws = off_time + round_up(static_cast<size_t>(N) * 4, 256);
+    // Cap the table at 8 GiB; larger batches run as waves.
+    const size_t ws_full = plan->feasible ? spdy_workspace_bytes(plan, N) : 0;
+    const size_t ws_one = plan->feasible ? spdy_workspace_bytes(plan, 1) : 0;
+    const size_t ws_cap = std::max<size_t>(ws_one, static_cast<size_t>(8) << 30);
+    const size_t ws_bytes = std::min(ws_full, ws_cap) / std::max<size_t>(ws_one, 1) * ws_one;
+    const size_t total = off_ws + ws_bytes;
+    if (total > plan->arena_bytes) {
+        if (plan->d_arena) {
+            SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
+            SPDY_CUDA_TRY(cudaFree(plan->d_arena));
+            plan->d_arena = nullptr;
+            plan->arena_bytes = 0;
+        }
+        cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&plan->d_arena), total);
+        if (err != cudaSuccess) {
+            g_last_cuda_error = static_cast<int>(err);
+            plan->d_arena = nullptr;
+            return err == cudaErrorMemoryAllocation ? SPDY_ERR_NO_MEMORY : SPDY_ERR_CUDA;
+        }
+        plan->arena_bytes = total;
+    }
+    unsigned char *base = plan->d_arena;
+    float *d_err = reinterpret_cast<float *>(base);
+    uint8_t *d_profile = base + off_profile;
+    float *d_cost = reinterpret_cast<float *>(base + off_cost);
+    int32_t *d_time = reinterpret_cast<int32_t *>(base + off_time);
+    SPDY_CUDA_TRY(cudaMemcpyAsync(d_err, errors_host, err_bytes, cudaMemcpyHostToDevice, stream));
+    rc = spdy_solve_batch(plan, d_err, N, d_profile, d_cost, d_time, base + off_ws, ws_bytes, stream);
+    if (rc != SPDY_OK) return rc;
+    SPDY_CUDA_TRY(cudaMemcpyAsync(profile_host, d_profile, static_cast<size_t>(N) * plan->L, cudaMemcpyDeviceToHost, stream));
+    SPDY_CUDA_TRY(cudaMemcpyAsync(cost_host, d_cost, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
+    SPDY_CUDA_TRY(cudaMemcpyAsync(time_used_host, d_time, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
+    SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
+    return SPDY_OK;
+}
+
+int spdy_solve_batch_simple(const float *errors_dev, const int32_t *times_dev, int64_t N,
+                            int32_t L, int32_t K, int32_t B, uint8_t *profile_dev, float *cost_dev,
+                            int32_t *time_used_dev, void *cuda_stream)
+{
+    if (!times_dev || L < 1 || K < 1 || K > 255 || B < 0 || N < 0) return SPDY_ERR_INVALID_ARG;
+    if (N == 0) return SPDY_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int device = 0;
+    SPDY_CUDA_TRY(cudaGetDevice(&device));
+    std::vector<int32_t> times;
+    try {
+        times.resize(static_cast<size_t>(L) * K);
+    } catch (const std::bad_alloc &) {
+        return SPDY_ERR_NO_MEMORY;
+    }
+    SPDY_CUDA_TRY(cudaMemcpyAsync(times.data(), times_dev, times.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
+    spdy_plan *plan = nullptr;
+    int rc = spdy_plan_create(&plan, times.data(), L, K, B, device, nullptr);
+    if (rc != SPDY_OK) return rc;
+    void *ws = nullptr;
+    size_t ws_bytes = 0;
+    if (plan->feasible) {
+        size_t free_b = 0, total_b = 0;
+        cudaError_t err = cudaMemGetInfo(&free_b, &total_b);
+        const size_t one = spdy_workspace_bytes(plan, 1);
+        const size_t want = spdy_workspace_bytes(plan, N);
+        ws_bytes = want;
+        if (err == cudaSuccess && want > free_b / 2) ws_bytes = std::max(one, (free_b / 2) / one * one);
+        err = cudaMalloc(&ws, ws_bytes);
+        if (err != cudaSuccess) {
+            g_last_cuda_error = static_cast<int>(err);
+            spdy_plan_destroy(plan);
+            return err == cudaErrorMemoryAllocation ? SPDY_ERR_NO_MEMORY : SPDY_ERR_CUDA;
+        }
+    }
+    rc = spdy_solve_batch(plan, errors_dev, N, profile_dev, cost_dev, time_used_dev, ws, ws_bytes, stream);
+    cudaError_t sync_err = cudaStreamSynchronize(stream);
+    if (rc == SPDY_OK && sync_err != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(sync_err);
+        rc = SPDY_ERR_CUDA;
+    }
+    if (rc == SPDY_OK) rc = spdy_plan_check_status(plan, stream);
+    if (ws) cudaFree(ws);
+    spdy_plan_destroy(plan);
+    return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,193 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle: bit-exact profiles, fp32 costs
+and time_used on the same seeded inputs."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2201_13096_b200 import binding, build as build_mod, workloads as W
+from helpers import check_solution
+
+pytestmark = pytest.mark.gpu
+
+FORMATS = [binding.SPDY_TABLE_ARG_U8, binding.SPDY_TABLE_ROW_F32]
+CORES = max(1, len(os.sched_getaffinity(0)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    build_mod.build()
+
+
+def gpu_solve(wl, fmt=0, **kw):
+    import torch
+
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt, **kw)
+    errors = torch.from_numpy(wl.errors).cuda()
+    p, c, t = binding.solve_batch(plan, errors)
+    torch.cuda.synchronize()
+    plan.check_status()
+    out = p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()
+    plan.close()
+    return out
+
+
+def assert_same(gpu, ref):
+    gp, gc, gt = gpu
+    rp, rc, rt = ref
+    assert np.array_equal(gt, rt), "time_used differs"
+    assert gc.tobytes() == rc.tobytes(), "cost bits differ"
+    assert np.array_equal(gp, rp), "profiles differ"
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_config0_many_seeds(fmt):
+    for seed in range(25):
+        wl = W.make_workload(0, seed_shift=seed)
+        assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B))
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("cfg,N", [(1, 96), (2, 96), (3, 6)])
+def test_named_configs_element_by_element(cfg, N, fmt):
+    wl = W.make_workload(cfg, N=N)
+    assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_sweep_budgets_of_config4(fmt):
+    for B, N in ((1000, 64), (10000, 16)):
+        wl = W.make_workload(4, N=N, B=B)
+        assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_adversarial_tiny_instances(fmt):
+    """Ties, zero times, times above the budget, +inf and negative errors, infeasible budgets."""
+    for seed in range(120):
+        for exact in (False, True):
+            wl = W.tiny_random_instance(seed + (10_000 if exact else 0), exact=exact, N=5)
+            assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B))
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_tie_heavy_wide_instance(fmt):
+    """Errors from {0, 1/4, 1/2, 1} and repeated / zero times on rows several spans wide."""
+    rng = np.random.default_rng(77)
+    L, K, B, N = 12, 9, 3000, 24
+    times = rng.integers(0, 400, size=(L, K)).astype(np.int32)
+    times[:, 3] = times[:, 2]
+    times[4, :] = 0
+    errors = rng.choice(np.array([0, 0.25, 0.5, 1.0], np.float32), size=(N, L, K)).astype(np.float32)
+    wl = W.Workload("ties", times, errors, B)
+    assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_paper_shaped_errors_of_eq4(fmt):
+    wl2 = W.make_workload(2, N=1)
+    errors = W.paper_shaped_errors(wl2.L, wl2.K, 48, seed=9)
+    wl = W.Workload("eq4", wl2.times, errors, wl2.B)
+    assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_degenerate_shapes(fmt):
+    import torch
+
+    cases = [
+        W.Workload("K1", np.array([[2], [0], [5]], np.int32), np.array([[[1.5], [2.5], [-0.25]]], np.float32), 7),
+        W.Workload("L1", np.array([[9, 7, 5, 5, 3, 11]], np.int32),
+                   np.array([[[0.0, 0.25, 0.5, 0.5, 2.0, -1.0]]], np.float32), 6),
+        W.Workload("B0", np.array([[0, 1], [0, 0]], np.int32), np.array([[[3.0, 1.0], [2.0, 2.0]]], np.float32), 0),
+        W.Workload("B0-infeasible", np.array([[1, 1]], np.int32), np.array([[[3.0, 1.0]]], np.float32), 0),
+        W.Workload("over", np.array([[50, 4], [60, 70]], np.int32), np.array([[[0.0, 1.0], [0.0, 1.0]]], np.float32), 10),
+        W.Workload("all-inf-layer", np.array([[1, 2], [1, 2]], np.int32),
+                   np.array([[[1.0, 2.0], [np.inf, np.inf]], [[1.0, 2.0], [3.0, np.inf]]], np.float32), 4),
+        W.Workload("neg-zero", np.array([[1, 2], [1, 2]], np.int32),
+                   np.array([[[-0.0, 2.0], [-0.0, 1.0]]], np.float32), 4),
+    ]
+    for wl in cases:
+        assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B))
+    # K = 255 (the largest choice count) and N = 0
+    rng = np.random.default_rng(1)
+    wl = W.Workload("K255", rng.integers(1, 40, size=(4, 255)).astype(np.int32),
+                    rng.lognormal(size=(3, 4, 255)).astype(np.float32), 90)
+    assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B))
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+    p, c, t = binding.solve_batch(plan, torch.empty((0, 4, 255), device="cuda"))
+    assert p.shape == (0, 4) and c.numel() == 0
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_small_workspace_runs_in_waves(fmt):
+    import torch
+
+    wl = W.make_workload(1, N=23)
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+    ws = torch.empty(plan.workspace_bytes(5), dtype=torch.uint8, device="cuda")
+    p, c, t = binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda(), workspace=ws)
+    torch.cuda.synchronize()
+    assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()),
+                oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+    tiny = torch.empty(plan.workspace_bytes(1) - 256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.SpdyError) as e:
+        binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda(), workspace=tiny)
+    assert e.value.status == -2
+    with pytest.raises(binding.SpdyError) as e:  # misaligned workspace
+        binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda(), workspace=ws[8:])
+    assert e.value.status == -1
+
+
+@pytest.mark.parametrize("threads", [128, 256, 512, 1024])
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_every_launch_shape_gives_the_same_answer(threads, fmt):
+    wl = W.make_workload(2, N=8)
+    assert_same(gpu_solve(wl, fmt, threads=threads), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+
+
+def test_host_buffer_and_one_shot_entry_points():
+    import torch
+
+    wl = W.make_workload(1, N=40)
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+    plan = binding.Plan(wl.times, wl.B, device=0)
+    assert_same(binding.solve_batch_host(plan, wl.errors), ref)
+    assert_same(binding.solve_batch_host(plan, wl.errors[:7]), tuple(x[:7] for x in ref))
+    pinned = torch.from_numpy(wl.errors).pin_memory()
+    assert_same(binding.solve_batch_host(plan, pinned), ref)
+    p, c, t = binding.solve_batch_simple(torch.from_numpy(wl.errors).cuda(), torch.from_numpy(wl.times).cuda(), wl.B)
+    assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), ref)
+    # a plan-level infeasible budget goes through the fill kernel
+    B_bad = int(wl.times.min(axis=1).sum()) - 1
+    p, c, t = binding.solve_batch_simple(torch.from_numpy(wl.errors).cuda(), torch.from_numpy(wl.times).cuda(), B_bad)
+    assert (p.cpu().numpy() == 0xFF).all() and (t.cpu().numpy() == -1).all() and np.isposinf(c.cpu().numpy()).all()
+
+
+def test_full_size_bert_base_batch_in_the_benchmark_configuration():
+    """N = 4096 as the benchmark times it: invariants on every candidate, oracle on a sample."""
+    import torch
+
+    wl = W.make_workload(2)
+    assert wl.N == 4096
+    plan = binding.Plan(wl.times, wl.B, device=0)
+    p, c, t = binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda())
+    torch.cuda.synchronize()
+    plan.check_status()
+    p, c, t = p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()
+    # invariants at full size (vectorised): total time and left-to-right fp32 sum of the profile
+    assert (t >= 0).all() and (t <= wl.B).all() and (p < wl.K).all()
+    idx = p.astype(np.int64)
+    tt = wl.times[np.arange(wl.L)[None, :], idx].sum(axis=1)
+    assert np.array_equal(tt, t)
+    e_sel = np.take_along_axis(wl.errors, idx[:, :, None], axis=2)[:, :, 0]
+    acc = np.zeros(wl.N, np.float32)
+    for l in range(wl.L):
+        acc = (acc + e_sel[:, l]).astype(np.float32)
+    assert acc.tobytes() == c.tobytes()
+    sample = np.random.default_rng(0).choice(wl.N, size=64, replace=False)
+    ref = oracle.solve_batch(wl.errors[sample], wl.times, wl.B, threads=CORES)
+    assert_same((p[sample], c[sample], t[sample]), ref)
+    for n in sample[:4]:
+        check_solution(wl.errors[n], wl.times, wl.B, p[n], c[n], int(t[n]))
