@@ -40,6 +40,7 @@ def parse_args():
     ap.add_argument("--budget", type=int, default=None, help="override B (config 4 sweep)")
     ap.add_argument("--table", default="default", choices=["default", "arg", "row"])
     ap.add_argument("--threads", type=int, default=0)
+    ap.add_argument("--mode", type=int, default=0, help="forward kernel variant (see spdy_options.forward_mode)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU work budget of the oracle legs")
@@ -56,7 +57,7 @@ def host_cores() -> int:
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
 
-    def __init__(self, index: int, period: float = 0.05):
+    def __init__(self, index: int, period: float = 0.01):
         self.index, self.period = index, period
         self.samples, self.reasons = [], set()
         self.max_mhz = None
@@ -202,7 +203,10 @@ def run_ours(args):
     wl = W.make_workload(args.config, N=n_per_rank, B=args.budget, start=rank * n_per_rank)
     assert np.array_equal(probe.times, wl.times)
     fmt = {"default": 0, "arg": 1, "row": 2}[args.table]
-    plan = binding.Plan(wl.times, wl.B, device=local_rank, table_format=fmt, threads=args.threads)
+    if args.mode:
+        fmt = 1 if args.mode in (1, 2) else 2
+    plan = binding.Plan(wl.times, wl.B, device=local_rank, table_format=fmt, threads=args.threads,
+                        forward_mode=args.mode)
     info = plan.info
     plan.enable_timing(True)
 

@@ -57,9 +57,13 @@ typedef enum spdy_table_format {
 
 typedef struct spdy_options {
     int32_t table_format;  /* spdy_table_format */
-    int32_t threads;       /* threads per CTA, 0 = choose; multiple of 32 in [64, 1024] */
+    int32_t threads;       /* threads per CTA, 0 = choose; one of 128, 256, 512, 1024 and >= K */
     int32_t cluster;       /* CTAs cooperating on one candidate, 0 = choose; 1, 2, 4 or 8 */
-    int32_t reserved[5];   /* must be 0 */
+    int32_t forward_mode;  /* 0 = choose.  Variants of the forward kernel's cell update, all with
+                              identical results, for measurement: 1 compare+select (ARG_U8),
+                              2 compare+predicated moves (ARG_U8), 3 fp32 minimum (ROW_F32),
+                              4 packed adds + 3-input minimum over choice pairs (ROW_F32) */
+    int32_t reserved[4];   /* must be 0 */
 } spdy_options;
 
 /* Facts about a plan: shapes, the launch shape chosen, and work counts for measurement. */
@@ -67,7 +71,7 @@ typedef struct spdy_plan_info {
     int32_t L, K, B;
     int32_t feasible;       /* 0: sum of per-layer minimum times exceeds B, every candidate is infeasible */
     int32_t max_width;      /* widest live band, in cells */
-    int32_t span;           /* cells one warp processes per pass */
+    int32_t span;           /* most cells one warp processes per pass */
     int32_t threads;        /* threads per CTA */
     int32_t cluster;        /* CTAs per candidate */
     int32_t table_format;   /* resolved spdy_table_format */

@@ -26,7 +26,8 @@ EXPORTS = (
 
 class SpdyOptions(ctypes.Structure):
     _fields_ = [("table_format", ctypes.c_int32), ("threads", ctypes.c_int32),
-                ("cluster", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
+                ("cluster", ctypes.c_int32), ("forward_mode", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 4)]
 
 
 class SpdyPlanInfo(ctypes.Structure):
@@ -118,13 +119,14 @@ class Plan:
     """``spdy_plan``: everything that depends only on ``times`` and ``B``."""
 
     def __init__(self, times, B: int, device: int = 0, table_format: int = SPDY_TABLE_DEFAULT,
-                 threads: int = 0, cluster: int = 0):
+                 threads: int = 0, cluster: int = 0, forward_mode: int = 0):
         lib = _load()
         t = np.ascontiguousarray(np.asarray(times), dtype=np.int32)
         if t.ndim != 2:
             raise ValueError("times must be [L][K]")
         self.L, self.K, self.B, self.device = int(t.shape[0]), int(t.shape[1]), int(B), int(device)
-        opts = SpdyOptions(table_format=table_format, threads=threads, cluster=cluster)
+        opts = SpdyOptions(table_format=table_format, threads=threads, cluster=cluster,
+                           forward_mode=forward_mode)
         handle = ctypes.c_void_p()
         _check(lib.spdy_plan_create(ctypes.byref(handle), t.ctypes.data_as(ctypes.c_void_p),
                                     self.L, self.K, self.B, self.device, ctypes.byref(opts)),

@@ -35,14 +35,28 @@ thread_local int g_last_cuda_error = 0;
 // Device-side layout
 // ----------------------------------------------------------------------------------------------
 
+constexpr int RMAX = 16;        // most band cells one lane owns in one pass
+constexpr int PAD = 32 * RMAX;  // +inf guard cells on either side of a shared-memory row
+
+// How the forward kernel forms a cell and what it stores for the walk back.
+enum ForwardMode {
+    MODE_ARG = 1,      // compare + two selects per cell, byte table of winning choices
+    MODE_ARG_PRED = 2, // compare + two predicated moves per cell, byte table
+    MODE_ROW = 3,      // value-only minimum, fp32 table of row values
+    MODE_ROW2 = 4      // value-only, two choices per step: packed f32x2 adds and 3-input minimum
+};
+
 // Row l (1-based; stored at index l-1) lives on the band [lo, lo + width).  A band cell is
-// addressed by t_rel = t - lo.  `rowoff` is where the row starts inside one candidate's table,
-// in cells, always a multiple of the span.
+// addressed by t_rel = t - lo.  Within a layer every warp pass covers 32*cpl consecutive cells
+// ("span"); `rowoff` is where the row starts inside one candidate's table, in cells.
 struct LayerDesc {
     int32_t width;
     uint32_t rowoff;
     int32_t lo;
-    int32_t mn;  // smallest usable time of the layer: lo_l = lo_{l-1} + mn
+    int32_t mn;      // smallest usable time of the layer: lo_l = lo_{l-1} + mn
+    int32_t cpl;     // cells per lane per pass, 1..RMAX
+    int32_t nspans;  // passes needed to cover the band: ceil(width / (32*cpl))
+    int32_t pad0, pad1;
 };
 
 // One (layer, choice) pair in band coordinates: the choice contributes to cells t_rel in [a, b]
@@ -67,20 +81,162 @@ struct FwdArgs {
 
 __device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
 
-// Cells a warp owns in one pass: SPAN = 32*R consecutive band cells, lane i taking cells
-// i, i+32, ... so that every shared-memory access is lane-consecutive (conflict-free) whatever
-// the shift.  Both row buffers carry SPAN cells of +inf on either side of the band: a warp whose
-// span only partly overlaps a choice's range then reads +inf for the cells outside it, and no
-// per-cell bounds check is needed.
+// Two independent round-to-nearest fp32 adds in one instruction: (x, y) += (e, e).
+__device__ __forceinline__ void add2_rn(float &x, float &y, unsigned long long e2)
+{
+    unsigned long long p, r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "f"(x), "f"(y));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(p), "l"(e2));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(x), "=f"(y) : "l"(r));
+}
+
+__device__ __forceinline__ unsigned long long splat2(float e)
+{
+    unsigned long long p;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(p) : "f"(e));
+    return p;
+}
+
+__device__ __forceinline__ float min3(float a, float b, float c)
+{
+    float m;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+    return m;
+}
+
+// One warp pass: the 32*RR band cells starting at s (lane i owns cells s + i, s + i + 32, ...),
+// so every shared-memory access is lane-consecutive (conflict-free) whatever the shift.  Both row
+// buffers carry PAD cells of +inf on either side of the band: a pass that only partly overlaps a
+// choice's range reads +inf for the cells outside it and needs no per-cell bounds check; a choice
+// that does not overlap the pass at all is skipped (or, when paired, pointed at the +inf pad).
 //
-// Table layouts (internal, only the walk-back kernel reads them):
-//   ARG:  one byte per cell; inside a span the byte of cell u = 32*j + lane sits at lane*R + j,
-//         so each lane writes its R bytes with 16-byte stores.
-//   !ARG: one float per cell in natural order.
-template <int R, bool ARG, int NT, int MINB>
+// `prev`/`cur` point at band cell 0 of the previous/new row; taps[k] = (a, b, bits of e, float k).
+template <int RR, int MODE>
+__device__ __forceinline__ void process_span(const float *__restrict__ prev, float *__restrict__ cur,
+                                             const int4 *__restrict__ taps, const int K, const int s,
+                                             const int lane, void *table_row)
+{
+    constexpr int SPANC = 32 * RR;
+    const float INF = pos_inf();
+    const float *base = prev + lane;
+    float best[RR];
+#pragma unroll
+    for (int j = 0; j < RR; ++j) best[j] = INF;
+
+    if constexpr (MODE == MODE_ROW2) {
+        int k = 0;
+#pragma unroll 1
+        for (; k + 1 < K; k += 2) {
+            const int4 ta = taps[k];
+            const int4 tb = taps[k + 1];
+            const bool ia = (s + SPANC > ta.x) && (s <= ta.y);
+            const bool ib = (s + SPANC > tb.x) && (s <= tb.y);
+            if (!(ia || ib)) continue;  // warp-uniform
+            const float *sa = base + (ia ? s - ta.x : -PAD);
+            const float *sb = base + (ib ? s - tb.x : -PAD);
+            const float ea = __int_as_float(ta.z), eb = __int_as_float(tb.z);
+            const unsigned long long ea2 = splat2(ea), eb2 = splat2(eb);
+#pragma unroll
+            for (int j = 0; j + 1 < RR; j += 2) {
+                float a0 = sa[j * 32], a1 = sa[(j + 1) * 32];
+                float b0 = sb[j * 32], b1 = sb[(j + 1) * 32];
+                add2_rn(a0, a1, ea2);
+                add2_rn(b0, b1, eb2);
+                best[j] = min3(best[j], a0, b0);
+                best[j + 1] = min3(best[j + 1], a1, b1);
+            }
+            if (RR & 1) {
+                const float a0 = __fadd_rn(sa[(RR - 1) * 32], ea);
+                const float b0 = __fadd_rn(sb[(RR - 1) * 32], eb);
+                best[RR - 1] = min3(best[RR - 1], a0, b0);
+            }
+        }
+        if (k < K) {
+            const int4 ta = taps[k];
+            if ((s + SPANC > ta.x) && (s <= ta.y)) {
+                const float *sa = base + (s - ta.x);
+                const float ea = __int_as_float(ta.z);
+#pragma unroll
+                for (int j = 0; j < RR; ++j) best[j] = fminf(best[j], __fadd_rn(sa[j * 32], ea));
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < RR; ++j) cur[s + j * 32 + lane] = best[j];
+        float *D = static_cast<float *>(table_row) + s + lane;
+#pragma unroll
+        for (int j = 0; j < RR; ++j) D[j * 32] = best[j];
+    } else if constexpr (MODE == MODE_ROW) {
+#pragma unroll 1
+        for (int k = 0; k < K; ++k) {
+            const int4 tp = taps[k];
+            if (!((s + SPANC > tp.x) && (s <= tp.y))) continue;
+            const float *src = base + (s - tp.x);
+            const float e = __int_as_float(tp.z);
+#pragma unroll
+            for (int j = 0; j < RR; ++j) best[j] = fminf(best[j], __fadd_rn(src[j * 32], e));
+        }
+#pragma unroll
+        for (int j = 0; j < RR; ++j) cur[s + j * 32 + lane] = best[j];
+        float *D = static_cast<float *>(table_row) + s + lane;
+#pragma unroll
+        for (int j = 0; j < RR; ++j) D[j * 32] = best[j];
+    } else if constexpr (MODE == MODE_ARG) {
+        int idx[RR];
+#pragma unroll
+        for (int j = 0; j < RR; ++j) idx[j] = 0xFF;
+#pragma unroll 1
+        for (int k = 0; k < K; ++k) {
+            const int4 tp = taps[k];
+            if (!((s + SPANC > tp.x) && (s <= tp.y))) continue;
+            const float *src = base + (s - tp.x);
+            const float e = __int_as_float(tp.z);
+#pragma unroll
+            for (int j = 0; j < RR; ++j) {
+                const float v = __fadd_rn(src[j * 32], e);
+                const bool better = v < best[j];  // strict: the lowest k keeps a tie
+                best[j] = better ? v : best[j];
+                idx[j] = better ? k : idx[j];
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < RR; ++j) cur[s + j * 32 + lane] = best[j];
+        unsigned char *P = static_cast<unsigned char *>(table_row) + s + lane;
+#pragma unroll
+        for (int j = 0; j < RR; ++j) P[j * 32] = static_cast<unsigned char>(idx[j]);
+    } else {  // MODE_ARG_PRED
+        float idxf[RR];
+#pragma unroll
+        for (int j = 0; j < RR; ++j) idxf[j] = 255.0f;
+#pragma unroll 1
+        for (int k = 0; k < K; ++k) {
+            const int4 tp = taps[k];
+            if (!((s + SPANC > tp.x) && (s <= tp.y))) continue;
+            const float *src = base + (s - tp.x);
+            const float e = __int_as_float(tp.z);
+            const float kf = __int_as_float(tp.w);
+#pragma unroll
+            for (int j = 0; j < RR; ++j) {
+                const float v = __fadd_rn(src[j * 32], e);
+                // x + (-0.0) == x for every x, so the predicated adds are exact moves.
+                asm("{ .reg .pred p; setp.lt.f32 p, %2, %0;\n\t"
+                    "@p add.rn.f32 %0, %2, 0f80000000;\n\t"
+                    "@p add.rn.f32 %1, %3, 0f80000000; }"
+                    : "+f"(best[j]), "+f"(idxf[j])
+                    : "f"(v), "f"(kf));
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < RR; ++j) cur[s + j * 32 + lane] = best[j];
+        unsigned char *P = static_cast<unsigned char *>(table_row) + s + lane;
+#pragma unroll
+        for (int j = 0; j < RR; ++j) P[j * 32] = static_cast<unsigned char>(static_cast<int>(idxf[j]));
+    }
+}
+
+template <int MODE, int NT, int MINB>
 __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs args)
 {
-    constexpr int SPAN = 32 * R;
+    constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *rows = reinterpret_cast<float *>(smem_raw);
     int4 *tap_buf = reinterpret_cast<int4 *>(rows + 2 * static_cast<size_t>(args.row_stride));
@@ -97,96 +253,55 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
 
     // Both buffers start as +inf everywhere; D_0 is +0 at t = 0 (Eq. 3 via a virtual row 0).
     for (int i = tid; i < 2 * args.row_stride; i += NT) rows[i] = INF;
-    if (tid < K) {
-        const TapRange tr = args.taps[tid];
-        tap_buf[tid] = make_int4(tr.a, tr.b, __float_as_int(err_n[tid]), 0);
+    for (int k = tid; k < K; k += NT) {
+        const TapRange tr = args.taps[k];
+        tap_buf[k] = make_int4(tr.a, tr.b, __float_as_int(err_n[k]), __float_as_int(static_cast<float>(k)));
     }
     __syncthreads();
-    if (tid == 0) rows[SPAN] = 0.0f;
+    if (tid == 0) rows[PAD] = 0.0f;
     __syncthreads();
 
     for (int l = 0; l < L; ++l) {
-        const float *prev = rows + (l & 1) * args.row_stride + SPAN;
-        float *cur = rows + ((l + 1) & 1) * args.row_stride + SPAN;
+        const float *prev = rows + (l & 1) * args.row_stride + PAD;
+        float *cur = rows + ((l + 1) & 1) * args.row_stride + PAD;
         const int4 *taps = tap_buf + (l & 1) * K;
         const LayerDesc ld = args.layers[l];
-        const int nspans = (ld.width + SPAN - 1) / SPAN;
 
         // Fetch the next layer's choices early; they are parked in shared memory after the pass.
+        // (NT >= K is guaranteed by the host, so one thread per choice suffices.)
         int4 next_tap = make_int4(0, -1, 0, 0);
         const bool have_next = (l + 1 < L) && (tid < K);
         if (have_next) {
             const TapRange tr = args.taps[(l + 1) * K + tid];
-            next_tap = make_int4(tr.a, tr.b, __float_as_int(err_n[(l + 1) * K + tid]), 0);
+            next_tap = make_int4(tr.a, tr.b, __float_as_int(err_n[(l + 1) * K + tid]),
+                                 __float_as_int(static_cast<float>(tid)));
         }
 
-        for (int span = warp; span < nspans; span += NWARPS) {
-            const int s = span * SPAN;
-            float best[R];
-            int idx[R];
-#pragma unroll
-            for (int j = 0; j < R; ++j) {
-                best[j] = INF;
-                idx[j] = 0xFF;
-            }
-            const float *prev_lane = prev + s + lane;
-#pragma unroll 1
-            for (int k = 0; k < K; ++k) {
-                const int4 tp = taps[k];
-                if (s + SPAN > tp.x && s <= tp.y) {  // warp-uniform
-                    const float *src = prev_lane - tp.x;
-                    const float e = __int_as_float(tp.z);
-#pragma unroll
-                    for (int j = 0; j < R; ++j) {
-                        const float v = __fadd_rn(src[j * 32], e);
-                        if (ARG) {
-                            const bool better = v < best[j];
-                            best[j] = better ? v : best[j];
-                            idx[j] = better ? k : idx[j];
-                        } else {
-                            best[j] = fminf(best[j], v);
-                        }
-                    }
-                }
-            }
-#pragma unroll
-            for (int j = 0; j < R; ++j) cur[s + j * 32 + lane] = best[j];
-            if (ARG) {
-                unsigned char *P = static_cast<unsigned char *>(args.table) +
-                                   (n_local * args.pitch + ld.rowoff + s);
-                if (R % 16 == 0) {
-#pragma unroll
-                    for (int q = 0; q < R / 16; ++q) {
-                        uint4 w;
-                        w.x = idx[16 * q + 0] | (idx[16 * q + 1] << 8) | (idx[16 * q + 2] << 16) | (idx[16 * q + 3] << 24);
-                        w.y = idx[16 * q + 4] | (idx[16 * q + 5] << 8) | (idx[16 * q + 6] << 16) | (idx[16 * q + 7] << 24);
-                        w.z = idx[16 * q + 8] | (idx[16 * q + 9] << 8) | (idx[16 * q + 10] << 16) | (idx[16 * q + 11] << 24);
-                        w.w = idx[16 * q + 12] | (idx[16 * q + 13] << 8) | (idx[16 * q + 14] << 16) | (idx[16 * q + 15] << 24);
-                        reinterpret_cast<uint4 *>(P + lane * R)[q] = w;
-                    }
-                } else {
-                    static_assert(R % 16 == 0 || R == 8, "R must be 8 or a multiple of 16");
-                    uint2 w;
-                    w.x = idx[0] | (idx[1] << 8) | (idx[2] << 16) | (idx[3] << 24);
-                    w.y = idx[4] | (idx[5] << 8) | (idx[6] << 16) | (idx[7] << 24);
-                    *reinterpret_cast<uint2 *>(P + lane * R) = w;
-                }
-            } else {
-                float *D = static_cast<float *>(args.table) + (n_local * args.pitch + ld.rowoff + s) + lane;
-#pragma unroll
-                for (int j = 0; j < R; ++j) D[j * 32] = best[j];
-            }
+        unsigned char *row_base = static_cast<unsigned char *>(args.table) +
+                                  (n_local * args.pitch + ld.rowoff) * (ROWFMT ? 4 : 1);
+        const int span_cells = 32 * ld.cpl;
+        switch (ld.cpl) {
+#define SPDY_CASE(RR)                                                                     \
+    case RR:                                                                              \
+        for (int span = warp; span < ld.nspans; span += NWARPS)                           \
+            process_span<RR, MODE>(prev, cur, taps, K, span * (32 * RR), lane, row_base); \
+        break;
+            SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
+            SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
+            SPDY_CASE(13) SPDY_CASE(14) SPDY_CASE(15) SPDY_CASE(16)
+#undef SPDY_CASE
+            default: break;
         }
-        // Cells [width, width + SPAN) of the new row must read as +inf for the next layer.  The
-        // spans above wrote +inf up to nspans*SPAN (their out-of-range cells saw only +inf
-        // sources); one more span of +inf covers the rest.
-        for (int i = tid; i < SPAN; i += NT) cur[nspans * SPAN + i] = INF;
+        // Cells [width, width + PAD) of the new row must read as +inf for the next layer.  The
+        // passes above wrote +inf from `width` up to nspans*span (those cells saw only +inf
+        // sources); PAD more cells of +inf cover the rest.
+        for (int i = tid; i < PAD; i += NT) cur[ld.nspans * span_cells + i] = INF;
         if (have_next) tap_buf[((l + 1) & 1) * K + tid] = next_tap;
         __syncthreads();
     }
 
     // min over t <= B of D_L[t], lowest t among equals (the band's upper end never exceeds B).
-    const float *last = rows + (L & 1) * args.row_stride + SPAN;
+    const float *last = rows + (L & 1) * args.row_stride + PAD;
     const LayerDesc ld = args.layers[L - 1];
     float bv = INF;
     int bt = 0x7fffffff;
@@ -245,7 +360,7 @@ struct BackArgs {
     int64_t pitch;
     int64_t n_first;
     int64_t n_count;
-    int32_t L, K, R;
+    int32_t L, K;
 };
 
 // Walk back through the byte table (end of Algorithm 1): one thread per candidate.
@@ -254,8 +369,7 @@ __global__ void spdy_backtrack_arg_kernel(const BackArgs args)
     const int64_t n_local = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
     if (n_local >= args.n_count) return;
     const int64_t n = args.n_first + n_local;
-    const int L = args.L, K = args.K, R = args.R;
-    const int span = 32 * R;
+    const int L = args.L, K = args.K;
     uint8_t *prof = args.profile + n * L;
     int t = args.time_used[n];
     if (t < 0) {
@@ -268,10 +382,7 @@ __global__ void spdy_backtrack_arg_kernel(const BackArgs args)
         const LayerDesc ld = args.layers[l];
         const int t_rel = t - ld.lo;
         int k = 0xFF;
-        if (ok && t_rel >= 0 && t_rel < ld.width) {
-            const int u = t_rel % span;
-            k = P[ld.rowoff + (t_rel - u) + (u & 31) * R + (u >> 5)];
-        }
+        if (ok && t_rel >= 0 && t_rel < ld.width) k = P[ld.rowoff + t_rel];
         if (k >= K) {
             ok = false;
             k = 0xFF;
@@ -374,30 +485,30 @@ __global__ void spdy_fill_infeasible_kernel(uint8_t *profile, float *cost, int32
 using FwdKernel = void (*)(const FwdArgs);
 
 struct FwdVariant {
-    int R;
-    bool arg;
+    int mode;
     int threads;
+    int min_blocks;
     FwdKernel fn;
 };
 
-#define SPDY_VARIANT(R, ARG, NT, MINB) \
-    FwdVariant { R, ARG, NT, spdy_forward_kernel<R, ARG, NT, MINB> }
+#define SPDY_VARIANT(MODE, NT, MINB) \
+    FwdVariant { MODE, NT, MINB, spdy_forward_kernel<MODE, NT, MINB> }
 
 const FwdVariant kVariants[] = {
-    SPDY_VARIANT(16, true, 128, 4),  SPDY_VARIANT(16, true, 256, 3),
-    SPDY_VARIANT(16, true, 512, 1),  SPDY_VARIANT(16, true, 1024, 1),
-    SPDY_VARIANT(16, false, 128, 4), SPDY_VARIANT(16, false, 256, 3),
-    SPDY_VARIANT(16, false, 512, 1), SPDY_VARIANT(16, false, 1024, 1),
-    SPDY_VARIANT(8, true, 128, 4),   SPDY_VARIANT(8, true, 256, 4),
-    SPDY_VARIANT(8, true, 512, 2),   SPDY_VARIANT(8, true, 1024, 1),
-    SPDY_VARIANT(8, false, 128, 4),  SPDY_VARIANT(8, false, 256, 4),
-    SPDY_VARIANT(8, false, 512, 2),  SPDY_VARIANT(8, false, 1024, 1),
+    SPDY_VARIANT(MODE_ARG, 128, 4),      SPDY_VARIANT(MODE_ARG, 256, 3),
+    SPDY_VARIANT(MODE_ARG, 512, 1),      SPDY_VARIANT(MODE_ARG, 1024, 1),
+    SPDY_VARIANT(MODE_ARG_PRED, 128, 4), SPDY_VARIANT(MODE_ARG_PRED, 256, 3),
+    SPDY_VARIANT(MODE_ARG_PRED, 512, 1), SPDY_VARIANT(MODE_ARG_PRED, 1024, 1),
+    SPDY_VARIANT(MODE_ROW, 128, 4),      SPDY_VARIANT(MODE_ROW, 256, 3),
+    SPDY_VARIANT(MODE_ROW, 512, 1),      SPDY_VARIANT(MODE_ROW, 1024, 1),
+    SPDY_VARIANT(MODE_ROW2, 128, 4),     SPDY_VARIANT(MODE_ROW2, 256, 3),
+    SPDY_VARIANT(MODE_ROW2, 512, 1),     SPDY_VARIANT(MODE_ROW2, 1024, 1),
 };
 
-const FwdVariant *find_variant(int R, bool arg, int threads)
+const FwdVariant *find_variant(int mode, int threads)
 {
     for (const FwdVariant &v : kVariants)
-        if (v.R == R && v.arg == arg && v.threads == threads) return &v;
+        if (v.mode == mode && v.threads == threads) return &v;
     return nullptr;
 }
 
@@ -413,7 +524,7 @@ struct spdy_plan {
     int32_t L = 0, K = 0, B = 0;
     int device = -1;
     bool feasible = false;
-    int R = 16;
+    int mode = MODE_ARG;
     int threads = 256;
     int cluster = 1;
     int table_format = SPDY_TABLE_ARG_U8;
@@ -507,28 +618,52 @@ int build_bands(spdy_plan *p)
     return SPDY_OK;
 }
 
-// Row offsets, table pitch and issued work for a given span.
-int layout_table(spdy_plan *p)
+// Per-layer pass shape for a CTA of `threads` threads, row offsets, table pitch and issued work.
+// A layer of `width` cells is covered in `rounds` rounds of NWARPS warp passes; the cells per lane
+// (cpl <= RMAX) are chosen so that the passes of a round are as full as possible, which keeps the
+// warps of a CTA level at the per-layer barrier.
+int layout_table(spdy_plan *p, int threads, double *efficiency)
 {
-    const int span = 32 * p->R;
-    int64_t off = 0;
+    const int nwarps = threads / 32;
+    int64_t off = 0, lanes_cells = 0;
+    int64_t max_extent = 0;
     p->issued_updates = 0;
     for (int l = 0; l < p->L; ++l) {
+        LayerDesc &ld = p->layers[l];
         if (off > 0xffffffffLL) return SPDY_ERR_UNSUPPORTED;
-        p->layers[l].rowoff = static_cast<uint32_t>(off);
-        const int64_t nspans = (p->layers[l].width + span - 1) / span;
-        off += nspans * span;
-        for (int k = 0; k < p->K; ++k) {
-            const TapRange tr = p->taps[static_cast<size_t>(l) * p->K + k];
-            if (tr.b < tr.a) continue;
-            const int64_t s_first = tr.a / span;  // first span whose end lies above a
-            const int64_t s_last = std::min<int64_t>(nspans - 1, tr.b / span);
-            if (s_last >= s_first) p->issued_updates += (s_last - s_first + 1) * span;
+        ld.rowoff = static_cast<uint32_t>(off);
+        const int64_t width = ld.width;
+        const int64_t per_round = 32LL * nwarps * RMAX;
+        const int64_t rounds = std::max<int64_t>(1, (width + per_round - 1) / per_round);
+        int64_t cpl = (width + 32LL * nwarps * rounds - 1) / (32LL * nwarps * rounds);
+        cpl = std::min<int64_t>(RMAX, std::max<int64_t>(1, cpl));
+        const int64_t span = 32 * cpl;
+        const int64_t nspans = (width + span - 1) / span;
+        ld.cpl = static_cast<int32_t>(cpl);
+        ld.nspans = static_cast<int32_t>(nspans);
+        max_extent = std::max(max_extent, nspans * span);
+        off += round_up(nspans * span, 128);
+        lanes_cells += ((nspans + nwarps - 1) / nwarps) * nwarps * span;
+        const bool paired = p->mode == MODE_ROW2;
+        for (int64_t sp = 0; sp < nspans; ++sp) {
+            const int64_t s = sp * span;
+            auto hits = [&](int k) {
+                const TapRange tr = p->taps[static_cast<size_t>(l) * p->K + k];
+                return tr.b >= tr.a && s + span > tr.a && s <= tr.b;
+            };
+            for (int k = 0; k < p->K; k += paired ? 2 : 1) {
+                if (paired && k + 1 < p->K) {
+                    if (hits(k) || hits(k + 1)) p->issued_updates += 2 * span;
+                } else if (hits(k)) {
+                    p->issued_updates += span;
+                }
+            }
         }
     }
     p->pitch = off;
-    p->row_stride = static_cast<int32_t>(round_up(p->max_width, span) + 2 * span);
+    p->row_stride = static_cast<int32_t>(round_up(max_extent, 32) + 2 * PAD);
     p->smem_bytes = 2LL * p->row_stride * 4 + 2LL * p->K * 16;
+    if (efficiency) *efficiency = lanes_cells > 0 ? static_cast<double>(p->band_cells) / lanes_cells : 0.0;
     return SPDY_OK;
 }
 
@@ -548,42 +683,51 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
     p->table_format = (opts && opts->table_format) ? opts->table_format : SPDY_TABLE_ARG_U8;
     if (p->table_format != SPDY_TABLE_ARG_U8 && p->table_format != SPDY_TABLE_ROW_F32)
         return SPDY_ERR_INVALID_ARG;
+    p->mode = p->table_format == SPDY_TABLE_ARG_U8 ? MODE_ARG : MODE_ROW2;
+    if (opts && opts->forward_mode) {
+        p->mode = opts->forward_mode;
+        const bool row_mode = p->mode == MODE_ROW || p->mode == MODE_ROW2;
+        const bool arg_mode = p->mode == MODE_ARG || p->mode == MODE_ARG_PRED;
+        if (!(row_mode || arg_mode)) return SPDY_ERR_INVALID_ARG;
+        if (row_mode != (p->table_format == SPDY_TABLE_ROW_F32)) return SPDY_ERR_INVALID_ARG;
+    }
     p->cluster = (opts && opts->cluster) ? opts->cluster : 1;
     if (p->cluster != 1) return SPDY_ERR_UNSUPPORTED;
 
-    p->R = 16;
-    int rc = layout_table(p);
-    if (rc != SPDY_OK) return rc;
-    if (p->smem_bytes > smem_per_block) {
-        p->R = 8;  // narrower guard bands
-        rc = layout_table(p);
+    // Candidate CTA sizes; keep the one whose rounds are fullest, preferring more resident warps.
+    const int sizes[] = {128, 256, 512, 1024};
+    int best_threads = 0;
+    double best_score = -1.0;
+    for (int threads : sizes) {
+        if (opts && opts->threads && opts->threads != threads) continue;
+        if (threads < p->K) continue;  // one thread per choice stages the next layer
+        double eff = 0.0;
+        int rc = layout_table(p, threads, &eff);
         if (rc != SPDY_OK) return rc;
-        if (p->smem_bytes > smem_per_block) return SPDY_ERR_UNSUPPORTED;
+        if (p->smem_bytes > smem_per_block) continue;
+        const int64_t by_smem = std::max<int64_t>(1, smem_per_sm / (p->smem_bytes + 1024));
+        const int64_t ctas = std::min<int64_t>(std::min<int64_t>(by_smem, 2048 / threads), 32);
+        const double warps = static_cast<double>(ctas * threads / 32);
+        // Below about 16 resident warps an SM cannot cover shared-memory latency.
+        const double score = eff * std::min(1.0, warps / 16.0) + 1e-3 * std::min(warps, 32.0) / 32.0;
+        if (score > best_score) {
+            best_score = score;
+            best_threads = threads;
+        }
     }
-    const int64_t by_smem = std::max<int64_t>(1, smem_per_sm / (p->smem_bytes + 1024));
-    int threads;
-    if (opts && opts->threads) {
-        threads = opts->threads;
-    } else if (by_smem >= 8) {
-        threads = 128;
-    } else if (by_smem >= 3) {
-        threads = 256;
-    } else if (by_smem == 2) {
-        threads = 512;
-    } else {
-        threads = 1024;
-    }
-    if (!(opts && opts->threads) && threads < p->K) threads = 256;  // one thread per choice stages the next layer
-    if (threads < p->K) return SPDY_ERR_INVALID_ARG;
-    p->threads = threads;
-    p->variant = find_variant(p->R, p->table_format == SPDY_TABLE_ARG_U8, threads);
+    if (best_threads == 0) return (opts && opts->threads) ? SPDY_ERR_INVALID_ARG : SPDY_ERR_UNSUPPORTED;
+    int rc = layout_table(p, best_threads, nullptr);
+    if (rc != SPDY_OK) return rc;
+    p->threads = best_threads;
+    p->variant = find_variant(p->mode, best_threads);
     if (!p->variant) return SPDY_ERR_INVALID_ARG;
-    p->ctas_per_sm = static_cast<int>(std::min<int64_t>(by_smem, 2048 / threads));
+    const int64_t by_smem = std::max<int64_t>(1, smem_per_sm / (p->smem_bytes + 1024));
+    p->ctas_per_sm = static_cast<int>(std::min<int64_t>(by_smem, 2048 / best_threads));
     if (p->device >= 0) {
         SPDY_CUDA_TRY(cudaFuncSetAttribute(p->variant->fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            static_cast<int>(p->smem_bytes)));
         int occ = 0;
-        SPDY_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, p->variant->fn, threads,
+        SPDY_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, p->variant->fn, best_threads,
                                                                     static_cast<size_t>(p->smem_bytes)));
         if (occ < 1) return SPDY_ERR_UNSUPPORTED;
         p->ctas_per_sm = occ;
@@ -663,9 +807,9 @@ int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int3
     *out = nullptr;
     if (!times_host || L < 1 || K < 1 || K > 255 || B < 0 || device < -1) return SPDY_ERR_INVALID_ARG;
     if (opts) {
-        for (int i = 0; i < 5; ++i)
+        for (int i = 0; i < 4; ++i)
             if (opts->reserved[i] != 0) return SPDY_ERR_INVALID_ARG;
-        if (opts->threads != 0 && (opts->threads % 32 != 0 || opts->threads < 64 || opts->threads > 1024))
+        if (opts->threads != 0 && (opts->threads % 32 != 0 || opts->threads < 32 || opts->threads > 1024))
             return SPDY_ERR_INVALID_ARG;
     }
     spdy_plan *p = new (std::nothrow) spdy_plan();
@@ -715,14 +859,14 @@ int spdy_plan_get_info(const spdy_plan *plan, spdy_plan_info *info)
     info->B = plan->B;
     info->feasible = plan->feasible ? 1 : 0;
     info->max_width = plan->max_width;
-    info->span = 32 * plan->R;
+    info->span = 32 * RMAX;
     info->threads = plan->threads;
     info->cluster = plan->cluster;
     info->table_format = plan->table_format;
     info->ctas_per_sm = plan->ctas_per_sm;
     info->sm_count = plan->sm_count;
     info->smem_bytes = plan->smem_bytes;
-    info->table_bytes_per_candidate = plan->pitch * cell_bytes(plan);
+    info->table_bytes_per_candidate = static_cast<int64_t>(spdy_workspace_bytes(plan, 1));
     info->band_cells = plan->band_cells;
     info->useful_updates = plan->useful_updates;
     info->issued_updates = plan->issued_updates;
@@ -820,7 +964,6 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
         ba.n_count = count;
         ba.L = plan->L;
         ba.K = plan->K;
-        ba.R = plan->R;
         if (plan->table_format == SPDY_TABLE_ARG_U8) {
             const int bt = 64;
             spdy_backtrack_arg_kernel<<<static_cast<unsigned>((count + bt - 1) / bt), bt, 0, stream>>>(ba);

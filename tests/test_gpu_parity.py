@@ -141,10 +141,15 @@ def test_small_workspace_runs_in_waves(fmt):
 
 
 @pytest.mark.parametrize("threads", [128, 256, 512, 1024])
-@pytest.mark.parametrize("fmt", FORMATS)
-def test_every_launch_shape_gives_the_same_answer(threads, fmt):
+@pytest.mark.parametrize("mode", [1, 2, 3, 4])
+def test_every_launch_shape_and_cell_update_variant_gives_the_same_answer(threads, mode):
     wl = W.make_workload(2, N=8)
-    assert_same(gpu_solve(wl, fmt, threads=threads), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+    fmt = 1 if mode in (1, 2) else 2
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+    assert_same(gpu_solve(wl, fmt, threads=threads, forward_mode=mode), ref)
+    tiny = W.tiny_random_instance(10_007, exact=True, N=5)
+    assert_same(gpu_solve(tiny, fmt, threads=threads, forward_mode=mode),
+                oracle.solve_batch(tiny.errors, tiny.times, tiny.B))
 
 
 def test_host_buffer_and_one_shot_entry_points():
