@@ -56,7 +56,8 @@ struct LayerDesc {
     int32_t mn;      // smallest usable time of the layer: lo_l = lo_{l-1} + mn
     int32_t cpl;     // cells per lane per pass, 1..RMAX
     int32_t nspans;  // passes needed to cover the band: ceil(width / (32*cpl))
-    int32_t pad0, pad1;
+    int32_t mask_off;  // index of the layer's first pass in the pass-mask table
+    int32_t pad1;
 };
 
 // One (layer, choice) pair in band coordinates: the choice contributes to cells t_rel in [a, b]
@@ -70,6 +71,8 @@ struct FwdArgs {
     const float *errors;      // [N][L][K]
     const TapRange *taps;     // [L][K]
     const LayerDesc *layers;  // [L]
+    const unsigned long long *span_masks;  // per pass: one bit per choice that overlaps it
+    const unsigned *span_kranges;          // per pass: k_lo | k_hi << 8 | dense << 16
     void *table;              // wave-local walk-back table
     float *cost;              // [N]
     int32_t *time_used;       // [N]
@@ -104,76 +107,131 @@ __device__ __forceinline__ float min3(float a, float b, float c)
     return m;
 }
 
+// Cell updates of one choice (or two) on the RR cells a lane owns; `sa`/`sb` point at the lane's
+// first source cell of the previous row, consecutive owned cells are 32 floats apart.
+template <int RR>
+__device__ __forceinline__ void update_min1(float (&best)[RR], const float *sa, const float ea)
+{
+#pragma unroll
+    for (int j = 0; j < RR; ++j) best[j] = fminf(best[j], __fadd_rn(sa[j * 32], ea));
+}
+
+template <int RR>
+__device__ __forceinline__ void update_min2(float (&best)[RR], const float *sa, const float ea,
+                                            const float *sb, const float eb)
+{
+    const unsigned long long ea2 = splat2(ea), eb2 = splat2(eb);
+#pragma unroll
+    for (int j = 0; j + 1 < RR; j += 2) {
+        float a0 = sa[j * 32], a1 = sa[(j + 1) * 32];
+        float b0 = sb[j * 32], b1 = sb[(j + 1) * 32];
+        add2_rn(a0, a1, ea2);
+        add2_rn(b0, b1, eb2);
+        best[j] = min3(best[j], a0, b0);
+        best[j + 1] = min3(best[j + 1], a1, b1);
+    }
+    if (RR & 1) {
+        const float a0 = __fadd_rn(sa[(RR - 1) * 32], ea);
+        const float b0 = __fadd_rn(sb[(RR - 1) * 32], eb);
+        best[RR - 1] = min3(best[RR - 1], a0, b0);
+    }
+}
+
+template <int RR>
+__device__ __forceinline__ void update_arg(float (&best)[RR], int (&idx)[RR], const float *src,
+                                           const float e, const int k)
+{
+#pragma unroll
+    for (int j = 0; j < RR; ++j) {
+        const float v = __fadd_rn(src[j * 32], e);
+        const bool better = v < best[j];  // strict: the lowest k keeps a tie
+        best[j] = better ? v : best[j];
+        idx[j] = better ? k : idx[j];
+    }
+}
+
+// Same update with the two selects written as predicated adds of -0.0 (x + (-0.0) == x for every
+// x, so they are exact moves) to keep them off the integer/compare pipe; the index is carried as
+// a float.
+template <int RR>
+__device__ __forceinline__ void update_arg_pred(float (&best)[RR], float (&idxf)[RR], const float *src,
+                                                const float e, const int k)
+{
+    const float kf = static_cast<float>(k);
+    const unsigned long long e2 = splat2(e);
+#define SPDY_PRED_UPDATE(J, V)                        \
+    asm("{ .reg .pred p; setp.lt.f32 p, %2, %0;\n\t"  \
+        "@p add.rn.f32 %0, %2, 0f80000000;\n\t"       \
+        "@p add.rn.f32 %1, %3, 0f80000000; }"         \
+        : "+f"(best[J]), "+f"(idxf[J])                \
+        : "f"(V), "f"(kf))
+#pragma unroll
+    for (int j = 0; j + 1 < RR; j += 2) {
+        float v0 = src[j * 32], v1 = src[(j + 1) * 32];
+        add2_rn(v0, v1, e2);
+        SPDY_PRED_UPDATE(j, v0);
+        SPDY_PRED_UPDATE(j + 1, v1);
+    }
+    if (RR & 1) {
+        const float v0 = __fadd_rn(src[(RR - 1) * 32], e);
+        SPDY_PRED_UPDATE(RR - 1, v0);
+    }
+#undef SPDY_PRED_UPDATE
+}
+
 // One warp pass: the 32*RR band cells starting at s (lane i owns cells s + i, s + i + 32, ...),
 // so every shared-memory access is lane-consecutive (conflict-free) whatever the shift.  Both row
 // buffers carry PAD cells of +inf on either side of the band: a pass that only partly overlaps a
-// choice's range reads +inf for the cells outside it and needs no per-cell bounds check; a choice
-// that does not overlap the pass at all is skipped (or, when paired, pointed at the +inf pad).
+// choice's range reads +inf for the cells outside it and needs no per-cell bounds check.  Which
+// choices overlap the pass at all is known on the host.  `krange` = k_lo | k_hi << 8 | dense << 16:
+// the overlapping choices lie in [k_lo, k_hi); when they are all of that range (dense, the usual
+// case: times fall as the choice index rises) the loop runs straight over it, otherwise it walks
+// the set bits of `mask` (MW 64-bit words, one bit per choice), in ascending order either way.
 //
-// `prev`/`cur` point at band cell 0 of the previous/new row; taps[k] = (a, b, bits of e, float k).
+// `prev`/`cur` point at band cell 0 of the previous/new row; taps[k] = (a_k, bits of e_k): choice
+// k reads the previous row at t_rel - a_k.
 template <int RR, int MODE>
 __device__ __forceinline__ void process_span(const float *__restrict__ prev, float *__restrict__ cur,
-                                             const int4 *__restrict__ taps, const int K, const int s,
-                                             const int lane, void *table_row)
+                                             const int2 *__restrict__ taps, const unsigned krange,
+                                             const unsigned long long *__restrict__ mask, const int MW,
+                                             const int s, const int lane, void *table_row)
 {
-    constexpr int SPANC = 32 * RR;
     const float INF = pos_inf();
-    const float *base = prev + lane;
+    const float *base = prev + s + lane;
+    const int k_lo = krange & 0xFF, k_hi = (krange >> 8) & 0xFF;
+    const bool dense = (krange >> 16) & 1;
     float best[RR];
 #pragma unroll
     for (int j = 0; j < RR; ++j) best[j] = INF;
 
-    if constexpr (MODE == MODE_ROW2) {
-        int k = 0;
+    if constexpr (MODE == MODE_ROW2 || MODE == MODE_ROW) {
+        // Value-only minimum: the order of the choices does not matter, so overlapping choices
+        // are taken two at a time (MODE_ROW2) whatever their indices.
+        if (dense) {
+            int k = k_lo;
+            if (MODE == MODE_ROW2) {
 #pragma unroll 1
-        for (; k + 1 < K; k += 2) {
-            const int4 ta = taps[k];
-            const int4 tb = taps[k + 1];
-            const bool ia = (s + SPANC > ta.x) && (s <= ta.y);
-            const bool ib = (s + SPANC > tb.x) && (s <= tb.y);
-            if (!(ia || ib)) continue;  // warp-uniform
-            const float *sa = base + (ia ? s - ta.x : -PAD);
-            const float *sb = base + (ib ? s - tb.x : -PAD);
-            const float ea = __int_as_float(ta.z), eb = __int_as_float(tb.z);
-            const unsigned long long ea2 = splat2(ea), eb2 = splat2(eb);
-#pragma unroll
-            for (int j = 0; j + 1 < RR; j += 2) {
-                float a0 = sa[j * 32], a1 = sa[(j + 1) * 32];
-                float b0 = sb[j * 32], b1 = sb[(j + 1) * 32];
-                add2_rn(a0, a1, ea2);
-                add2_rn(b0, b1, eb2);
-                best[j] = min3(best[j], a0, b0);
-                best[j + 1] = min3(best[j + 1], a1, b1);
+                for (; k + 1 < k_hi; k += 2) {
+                    const int2 ta = taps[k], tb = taps[k + 1];
+                    update_min2<RR>(best, base - ta.x, __int_as_float(ta.y), base - tb.x, __int_as_float(tb.y));
+                }
             }
-            if (RR & 1) {
-                const float a0 = __fadd_rn(sa[(RR - 1) * 32], ea);
-                const float b0 = __fadd_rn(sb[(RR - 1) * 32], eb);
-                best[RR - 1] = min3(best[RR - 1], a0, b0);
-            }
-        }
-        if (k < K) {
-            const int4 ta = taps[k];
-            if ((s + SPANC > ta.x) && (s <= ta.y)) {
-                const float *sa = base + (s - ta.x);
-                const float ea = __int_as_float(ta.z);
-#pragma unroll
-                for (int j = 0; j < RR; ++j) best[j] = fminf(best[j], __fadd_rn(sa[j * 32], ea));
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < RR; ++j) cur[s + j * 32 + lane] = best[j];
-        float *D = static_cast<float *>(table_row) + s + lane;
-#pragma unroll
-        for (int j = 0; j < RR; ++j) D[j * 32] = best[j];
-    } else if constexpr (MODE == MODE_ROW) {
 #pragma unroll 1
-        for (int k = 0; k < K; ++k) {
-            const int4 tp = taps[k];
-            if (!((s + SPANC > tp.x) && (s <= tp.y))) continue;
-            const float *src = base + (s - tp.x);
-            const float e = __int_as_float(tp.z);
-#pragma unroll
-            for (int j = 0; j < RR; ++j) best[j] = fminf(best[j], __fadd_rn(src[j * 32], e));
+            for (; k < k_hi; ++k) {
+                const int2 ta = taps[k];
+                update_min1<RR>(best, base - ta.x, __int_as_float(ta.y));
+            }
+        } else {
+#pragma unroll 1
+            for (int w = 0; w < MW; ++w) {
+                unsigned long long m = __ldg(mask + w);
+#pragma unroll 1
+                while (m) {
+                    const int2 ta = taps[64 * w + __ffsll(static_cast<long long>(m)) - 1];
+                    m &= m - 1;
+                    update_min1<RR>(best, base - ta.x, __int_as_float(ta.y));
+                }
+            }
         }
 #pragma unroll
         for (int j = 0; j < RR; ++j) cur[s + j * 32 + lane] = best[j];
@@ -184,18 +242,23 @@ __device__ __forceinline__ void process_span(const float *__restrict__ prev, flo
         int idx[RR];
 #pragma unroll
         for (int j = 0; j < RR; ++j) idx[j] = 0xFF;
+        if (dense) {
 #pragma unroll 1
-        for (int k = 0; k < K; ++k) {
-            const int4 tp = taps[k];
-            if (!((s + SPANC > tp.x) && (s <= tp.y))) continue;
-            const float *src = base + (s - tp.x);
-            const float e = __int_as_float(tp.z);
-#pragma unroll
-            for (int j = 0; j < RR; ++j) {
-                const float v = __fadd_rn(src[j * 32], e);
-                const bool better = v < best[j];  // strict: the lowest k keeps a tie
-                best[j] = better ? v : best[j];
-                idx[j] = better ? k : idx[j];
+            for (int k = k_lo; k < k_hi; ++k) {
+                const int2 tp = taps[k];
+                update_arg<RR>(best, idx, base - tp.x, __int_as_float(tp.y), k);
+            }
+        } else {
+#pragma unroll 1
+            for (int w = 0; w < MW; ++w) {
+                unsigned long long m = __ldg(mask + w);
+#pragma unroll 1
+                while (m) {
+                    const int k = 64 * w + __ffsll(static_cast<long long>(m)) - 1;
+                    m &= m - 1;
+                    const int2 tp = taps[k];
+                    update_arg<RR>(best, idx, base - tp.x, __int_as_float(tp.y), k);
+                }
             }
         }
 #pragma unroll
@@ -207,22 +270,23 @@ __device__ __forceinline__ void process_span(const float *__restrict__ prev, flo
         float idxf[RR];
 #pragma unroll
         for (int j = 0; j < RR; ++j) idxf[j] = 255.0f;
+        if (dense) {
 #pragma unroll 1
-        for (int k = 0; k < K; ++k) {
-            const int4 tp = taps[k];
-            if (!((s + SPANC > tp.x) && (s <= tp.y))) continue;
-            const float *src = base + (s - tp.x);
-            const float e = __int_as_float(tp.z);
-            const float kf = __int_as_float(tp.w);
-#pragma unroll
-            for (int j = 0; j < RR; ++j) {
-                const float v = __fadd_rn(src[j * 32], e);
-                // x + (-0.0) == x for every x, so the predicated adds are exact moves.
-                asm("{ .reg .pred p; setp.lt.f32 p, %2, %0;\n\t"
-                    "@p add.rn.f32 %0, %2, 0f80000000;\n\t"
-                    "@p add.rn.f32 %1, %3, 0f80000000; }"
-                    : "+f"(best[j]), "+f"(idxf[j])
-                    : "f"(v), "f"(kf));
+            for (int k = k_lo; k < k_hi; ++k) {
+                const int2 tp = taps[k];
+                update_arg_pred<RR>(best, idxf, base - tp.x, __int_as_float(tp.y), k);
+            }
+        } else {
+#pragma unroll 1
+            for (int w = 0; w < MW; ++w) {
+                unsigned long long m = __ldg(mask + w);
+#pragma unroll 1
+                while (m) {
+                    const int k = 64 * w + __ffsll(static_cast<long long>(m)) - 1;
+                    m &= m - 1;
+                    const int2 tp = taps[k];
+                    update_arg_pred<RR>(best, idxf, base - tp.x, __int_as_float(tp.y), k);
+                }
             }
         }
 #pragma unroll
@@ -239,7 +303,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
     constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *rows = reinterpret_cast<float *>(smem_raw);
-    int4 *tap_buf = reinterpret_cast<int4 *>(rows + 2 * static_cast<size_t>(args.row_stride));
+    int2 *tap_buf = reinterpret_cast<int2 *>(rows + 2 * static_cast<size_t>(args.row_stride));
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -253,10 +317,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
 
     // Both buffers start as +inf everywhere; D_0 is +0 at t = 0 (Eq. 3 via a virtual row 0).
     for (int i = tid; i < 2 * args.row_stride; i += NT) rows[i] = INF;
-    for (int k = tid; k < K; k += NT) {
-        const TapRange tr = args.taps[k];
-        tap_buf[k] = make_int4(tr.a, tr.b, __float_as_int(err_n[k]), __float_as_int(static_cast<float>(k)));
-    }
+    for (int k = tid; k < K; k += NT) tap_buf[k] = make_int2(args.taps[k].a, __float_as_int(err_n[k]));
     __syncthreads();
     if (tid == 0) rows[PAD] = 0.0f;
     __syncthreads();
@@ -264,27 +325,28 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
     for (int l = 0; l < L; ++l) {
         const float *prev = rows + (l & 1) * args.row_stride + PAD;
         float *cur = rows + ((l + 1) & 1) * args.row_stride + PAD;
-        const int4 *taps = tap_buf + (l & 1) * K;
+        const int2 *taps = tap_buf + (l & 1) * K;
         const LayerDesc ld = args.layers[l];
 
         // Fetch the next layer's choices early; they are parked in shared memory after the pass.
         // (NT >= K is guaranteed by the host, so one thread per choice suffices.)
-        int4 next_tap = make_int4(0, -1, 0, 0);
+        int2 next_tap = make_int2(0, 0);
         const bool have_next = (l + 1 < L) && (tid < K);
-        if (have_next) {
-            const TapRange tr = args.taps[(l + 1) * K + tid];
-            next_tap = make_int4(tr.a, tr.b, __float_as_int(err_n[(l + 1) * K + tid]),
-                                 __float_as_int(static_cast<float>(tid)));
-        }
+        if (have_next)
+            next_tap = make_int2(args.taps[(l + 1) * K + tid].a, __float_as_int(err_n[(l + 1) * K + tid]));
 
         unsigned char *row_base = static_cast<unsigned char *>(args.table) +
                                   (n_local * args.pitch + ld.rowoff) * (ROWFMT ? 4 : 1);
         const int span_cells = 32 * ld.cpl;
+        const int MW = (K + 63) >> 6;
+        const unsigned long long *masks = args.span_masks + static_cast<size_t>(ld.mask_off) * MW;
+        const unsigned *kranges = args.span_kranges + ld.mask_off;
         switch (ld.cpl) {
-#define SPDY_CASE(RR)                                                                     \
-    case RR:                                                                              \
-        for (int span = warp; span < ld.nspans; span += NWARPS)                           \
-            process_span<RR, MODE>(prev, cur, taps, K, span * (32 * RR), lane, row_base); \
+#define SPDY_CASE(RR)                                                                          \
+    case RR:                                                                                   \
+        for (int span = warp; span < ld.nspans; span += NWARPS)                                \
+            process_span<RR, MODE>(prev, cur, taps, __ldg(kranges + span), masks + span * MW,  \
+                                   MW, span * (32 * RR), lane, row_base);                      \
         break;
             SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
             SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
@@ -538,12 +600,16 @@ struct spdy_plan {
     std::vector<int32_t> times;
     std::vector<LayerDesc> layers;
     std::vector<TapRange> taps;
+    std::vector<uint64_t> span_masks;
+    std::vector<uint32_t> span_kranges;
     const FwdVariant *variant = nullptr;
     // device tables (one allocation)
     unsigned char *d_blob = nullptr;
     int32_t *d_times = nullptr;
     LayerDesc *d_layers = nullptr;
     TapRange *d_taps = nullptr;
+    unsigned long long *d_masks = nullptr;
+    unsigned *d_kranges = nullptr;
     int32_t *d_status = nullptr;
     // optional event timing of the last solve (three events per wave)
     bool timing = false;
@@ -625,6 +691,9 @@ int build_bands(spdy_plan *p)
 int layout_table(spdy_plan *p, int threads, double *efficiency)
 {
     const int nwarps = threads / 32;
+    const int mw = (p->K + 63) / 64;
+    p->span_masks.clear();
+    p->span_kranges.clear();
     int64_t off = 0, lanes_cells = 0;
     int64_t max_extent = 0;
     p->issued_updates = 0;
@@ -644,25 +713,33 @@ int layout_table(spdy_plan *p, int threads, double *efficiency)
         max_extent = std::max(max_extent, nspans * span);
         off += round_up(nspans * span, 128);
         lanes_cells += ((nspans + nwarps - 1) / nwarps) * nwarps * span;
-        const bool paired = p->mode == MODE_ROW2;
+        ld.mask_off = static_cast<int32_t>(p->span_masks.size() / mw);
         for (int64_t sp = 0; sp < nspans; ++sp) {
             const int64_t s = sp * span;
-            auto hits = [&](int k) {
+            uint64_t words[4] = {0, 0, 0, 0};
+            for (int k = 0; k < p->K; ++k) {
                 const TapRange tr = p->taps[static_cast<size_t>(l) * p->K + k];
-                return tr.b >= tr.a && s + span > tr.a && s <= tr.b;
-            };
-            for (int k = 0; k < p->K; k += paired ? 2 : 1) {
-                if (paired && k + 1 < p->K) {
-                    if (hits(k) || hits(k + 1)) p->issued_updates += 2 * span;
-                } else if (hits(k)) {
+                if (tr.b >= tr.a && s + span > tr.a && s <= tr.b) {
+                    words[k >> 6] |= 1ULL << (k & 63);
                     p->issued_updates += span;
                 }
             }
+            for (int w = 0; w < mw; ++w) p->span_masks.push_back(words[w]);
+            int k_lo = 0, k_hi = 0, count = 0;
+            for (int k = 0; k < p->K; ++k) {
+                if (words[k >> 6] >> (k & 63) & 1) {
+                    if (count == 0) k_lo = k;
+                    k_hi = k + 1;
+                    ++count;
+                }
+            }
+            const uint32_t dense = (count == k_hi - k_lo) ? 1u : 0u;
+            p->span_kranges.push_back(static_cast<uint32_t>(k_lo) | static_cast<uint32_t>(k_hi) << 8 | dense << 16);
         }
     }
     p->pitch = off;
     p->row_stride = static_cast<int32_t>(round_up(max_extent, 32) + 2 * PAD);
-    p->smem_bytes = 2LL * p->row_stride * 4 + 2LL * p->K * 16;
+    p->smem_bytes = 2LL * p->row_stride * 4 + 2LL * p->K * 8;
     if (efficiency) *efficiency = lanes_cells > 0 ? static_cast<double>(p->band_cells) / lanes_cells : 0.0;
     return SPDY_OK;
 }
@@ -740,12 +817,18 @@ int upload_tables(spdy_plan *p)
     const size_t n_times = static_cast<size_t>(p->L) * p->K;
     const size_t off_layers = round_up(n_times * sizeof(int32_t), 256);
     const size_t off_taps = off_layers + round_up(p->L * sizeof(LayerDesc), 256);
-    const size_t off_status = off_taps + round_up(n_times * sizeof(TapRange), 256);
+    const size_t off_masks = off_taps + round_up(n_times * sizeof(TapRange), 256);
+    const size_t off_kranges = off_masks + round_up(p->span_masks.size() * sizeof(uint64_t) + 8, 256);
+    const size_t off_status = off_kranges + round_up(p->span_kranges.size() * sizeof(uint32_t) + 4, 256);
     const size_t total = off_status + 256;
     std::vector<unsigned char> host(total, 0);
     std::memcpy(host.data(), p->times.data(), n_times * sizeof(int32_t));
     std::memcpy(host.data() + off_layers, p->layers.data(), p->L * sizeof(LayerDesc));
     std::memcpy(host.data() + off_taps, p->taps.data(), n_times * sizeof(TapRange));
+    if (!p->span_masks.empty())
+        std::memcpy(host.data() + off_masks, p->span_masks.data(), p->span_masks.size() * sizeof(uint64_t));
+    if (!p->span_kranges.empty())
+        std::memcpy(host.data() + off_kranges, p->span_kranges.data(), p->span_kranges.size() * sizeof(uint32_t));
     cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&p->d_blob), total);
     if (err != cudaSuccess) {
         g_last_cuda_error = static_cast<int>(err);
@@ -756,6 +839,8 @@ int upload_tables(spdy_plan *p)
     p->d_times = reinterpret_cast<int32_t *>(p->d_blob);
     p->d_layers = reinterpret_cast<LayerDesc *>(p->d_blob + off_layers);
     p->d_taps = reinterpret_cast<TapRange *>(p->d_blob + off_taps);
+    p->d_masks = reinterpret_cast<unsigned long long *>(p->d_blob + off_masks);
+    p->d_kranges = reinterpret_cast<unsigned *>(p->d_blob + off_kranges);
     p->d_status = reinterpret_cast<int32_t *>(p->d_blob + off_status);
     return SPDY_OK;
 }
@@ -937,6 +1022,8 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
         fa.errors = errors_dev;
         fa.taps = plan->d_taps;
         fa.layers = plan->d_layers;
+        fa.span_masks = plan->d_masks;
+        fa.span_kranges = plan->d_kranges;
         fa.table = workspace_dev;
         fa.cost = cost_dev;
         fa.time_used = time_used_dev;
