@@ -150,9 +150,9 @@ __device__ __forceinline__ void update_arg(float (&best)[RR], int (&idx)[RR], co
     }
 }
 
-// Same update with the two selects written as predicated adds of -0.0 (x + (-0.0) == x for every
-// x, so they are exact moves) to keep them off the integer/compare pipe; the index is carried as
-// a float.
+// Same update with the two selects written as predicated fp32 arithmetic that acts as an exact
+// move, to keep them off the integer/compare pipe: best <- v + (-0.0) (== v for every v) and
+// idx <- v * 0 + k (== k: a winning v is finite, so v * 0 is +-0).  The index is carried as a float.
 template <int RR>
 __device__ __forceinline__ void update_arg_pred(float (&best)[RR], float (&idxf)[RR], const float *src,
                                                 const float e, const int k)
@@ -162,7 +162,7 @@ __device__ __forceinline__ void update_arg_pred(float (&best)[RR], float (&idxf)
 #define SPDY_PRED_UPDATE(J, V)                        \
     asm("{ .reg .pred p; setp.lt.f32 p, %2, %0;\n\t"  \
         "@p add.rn.f32 %0, %2, 0f80000000;\n\t"       \
-        "@p add.rn.f32 %1, %3, 0f80000000; }"         \
+        "@p fma.rn.f32 %1, %2, 0f00000000, %3; }"     \
         : "+f"(best[J]), "+f"(idxf[J])                \
         : "f"(V), "f"(kf))
 #pragma unroll
@@ -589,7 +589,7 @@ struct spdy_plan {
     int mode = MODE_ARG;
     int threads = 256;
     int cluster = 1;
-    int table_format = SPDY_TABLE_ARG_U8;
+    int table_format = SPDY_TABLE_ROW_F32;
     int ctas_per_sm = 0;
     int sm_count = 148;
     int64_t smem_bytes = 0;
@@ -757,10 +757,10 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
         SPDY_CUDA_TRY(cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, p->device));
         p->sm_count = v;
     }
-    p->table_format = (opts && opts->table_format) ? opts->table_format : SPDY_TABLE_ARG_U8;
+    p->table_format = (opts && opts->table_format) ? opts->table_format : SPDY_TABLE_ROW_F32;
     if (p->table_format != SPDY_TABLE_ARG_U8 && p->table_format != SPDY_TABLE_ROW_F32)
         return SPDY_ERR_INVALID_ARG;
-    p->mode = p->table_format == SPDY_TABLE_ARG_U8 ? MODE_ARG : MODE_ROW2;
+    p->mode = p->table_format == SPDY_TABLE_ARG_U8 ? MODE_ARG_PRED : MODE_ROW2;
     if (opts && opts->forward_mode) {
         p->mode = opts->forward_mode;
         const bool row_mode = p->mode == MODE_ROW || p->mode == MODE_ROW2;
