@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--table", default="default", choices=["default", "arg", "row"])
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--mode", type=int, default=0, help="forward kernel variant (see spdy_options.forward_mode)")
+    ap.add_argument("--cluster", type=int, default=0, help="CTAs per candidate (0 = plan's choice)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU work budget of the oracle legs")
@@ -206,7 +207,7 @@ def run_ours(args):
     if args.mode:
         fmt = 1 if args.mode in (1, 2) else 2
     plan = binding.Plan(wl.times, wl.B, device=local_rank, table_format=fmt, threads=args.threads,
-                        forward_mode=args.mode)
+                        forward_mode=args.mode, cluster=args.cluster)
     info = plan.info
     plan.enable_timing(True)
 
@@ -315,6 +316,7 @@ def run_ours(args):
                    "timing": "sum of per-step CUDA-event pairs on the launch stream, max over ranks",
                    "table_format": {1: "arg_u8", 2: "row_f32"}[info["table_format"]],
                    "threads": info["threads"], "ctas_per_sm": info["ctas_per_sm"], "span": info["span"],
+                   "cluster": info["cluster"],
                    "waves": int(waves)},
         "nominal_cell_updates_per_s": cand_per_s * info["nominal_updates"],
         "useful_cell_updates_per_s": cand_per_s * info["useful_updates"],

@@ -10,6 +10,7 @@
 // results equal a plain sequential evaluation of Algorithm 1 with Eq. 2's bucket range.
 #include "../../include/spdy_dp.h"
 
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -190,11 +191,15 @@ __device__ __forceinline__ void update_arg_pred(float (&best)[RR], float (&idxf)
 //
 // `prev`/`cur` point at band cell 0 of the previous/new row; taps[k] = (a_k, bits of e_k): choice
 // k reads the previous row at t_rel - a_k.
-template <int RR, int MODE>
+//
+// With MASKED only cells below `limit` are stored (a CTA of a cluster owns a slice of the band and
+// must not write its neighbour's cells); without it the caller guarantees room for the whole pass.
+template <int RR, int MODE, bool MASKED>
 __device__ __forceinline__ void process_span(const float *__restrict__ prev, float *__restrict__ cur,
                                              const int2 *__restrict__ taps, const unsigned krange,
                                              const unsigned long long *__restrict__ mask, const int MW,
-                                             const int s, const int lane, void *table_row)
+                                             const int s, const int lane, void *table_row,
+                                             const int limit)
 {
     const float INF = pos_inf();
     const float *base = prev + s + lane;
@@ -234,10 +239,12 @@ __device__ __forceinline__ void process_span(const float *__restrict__ prev, flo
             }
         }
 #pragma unroll
-        for (int j = 0; j < RR; ++j) cur[s + j * 32 + lane] = best[j];
+        for (int j = 0; j < RR; ++j)
+            if (!MASKED || s + j * 32 + lane < limit) cur[s + j * 32 + lane] = best[j];
         float *D = static_cast<float *>(table_row) + s + lane;
 #pragma unroll
-        for (int j = 0; j < RR; ++j) D[j * 32] = best[j];
+        for (int j = 0; j < RR; ++j)
+            if (!MASKED || s + j * 32 + lane < limit) D[j * 32] = best[j];
     } else if constexpr (MODE == MODE_ARG) {
         int idx[RR];
 #pragma unroll
@@ -262,10 +269,12 @@ __device__ __forceinline__ void process_span(const float *__restrict__ prev, flo
             }
         }
 #pragma unroll
-        for (int j = 0; j < RR; ++j) cur[s + j * 32 + lane] = best[j];
+        for (int j = 0; j < RR; ++j)
+            if (!MASKED || s + j * 32 + lane < limit) cur[s + j * 32 + lane] = best[j];
         unsigned char *P = static_cast<unsigned char *>(table_row) + s + lane;
 #pragma unroll
-        for (int j = 0; j < RR; ++j) P[j * 32] = static_cast<unsigned char>(idx[j]);
+        for (int j = 0; j < RR; ++j)
+            if (!MASKED || s + j * 32 + lane < limit) P[j * 32] = static_cast<unsigned char>(idx[j]);
     } else {  // MODE_ARG_PRED
         float idxf[RR];
 #pragma unroll
@@ -290,10 +299,13 @@ __device__ __forceinline__ void process_span(const float *__restrict__ prev, flo
             }
         }
 #pragma unroll
-        for (int j = 0; j < RR; ++j) cur[s + j * 32 + lane] = best[j];
+        for (int j = 0; j < RR; ++j)
+            if (!MASKED || s + j * 32 + lane < limit) cur[s + j * 32 + lane] = best[j];
         unsigned char *P = static_cast<unsigned char *>(table_row) + s + lane;
 #pragma unroll
-        for (int j = 0; j < RR; ++j) P[j * 32] = static_cast<unsigned char>(static_cast<int>(idxf[j]));
+        for (int j = 0; j < RR; ++j)
+            if (!MASKED || s + j * 32 + lane < limit)
+                P[j * 32] = static_cast<unsigned char>(static_cast<int>(idxf[j]));
     }
 }
 
@@ -345,8 +357,9 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
 #define SPDY_CASE(RR)                                                                          \
     case RR:                                                                                   \
         for (int span = warp; span < ld.nspans; span += NWARPS)                                \
-            process_span<RR, MODE>(prev, cur, taps, __ldg(kranges + span), masks + span * MW,  \
-                                   MW, span * (32 * RR), lane, row_base);                      \
+            process_span<RR, MODE, false>(prev, cur, taps, __ldg(kranges + span),              \
+                                          masks + span * MW, MW, span * (32 * RR), lane,       \
+                                          row_base, 0);                                        \
         break;
             SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
             SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
@@ -407,6 +420,201 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
             args.cost[n] = feasible ? bv : INF;
             args.time_used[n] = feasible ? ld.lo + bt : -1;
         }
+    }
+}
+
+// ----------------------------------------------------------------------------------------------
+// Cluster variant: one candidate per thread-block cluster
+// ----------------------------------------------------------------------------------------------
+//
+// When two band-limited rows do not fit one CTA's shared memory (or when there are fewer
+// candidates than SMs) the band of every row is cut into C contiguous slices, one per CTA of a
+// cluster.  Each CTA keeps its slice of the new row in its own shared memory (`out`, double
+// buffered) and, before a layer, gathers the window of the previous row its slice depends on -
+// its own slice plus up to max_k a_k cells to the left - from the `out` buffers of its cluster
+// peers through distributed shared memory into a private window (`win`).  The cell updates then
+// run on local shared memory exactly as in the single-CTA kernel.  One hardware cluster barrier
+// per layer orders "slices of row l written" before "windows for row l+1 gathered"; every thread
+// of every CTA reaches every barrier (there is no early exit), so the barrier cannot wait forever.
+
+// Per (layer, rank) pass shape.  q0 is the first previous-row cell of the window.
+struct SliceDesc {
+    int32_t slice_lo;   // first band cell of the slice
+    int32_t slice_hi;   // one past the last (slice_lo == slice_hi: empty)
+    int32_t cpl;        // cells per lane per pass
+    int32_t nspans;     // passes covering the slice
+    int32_t mask_off;   // first pass in the pass tables
+    int32_t q0;         // first previous-row cell the passes may read
+    int32_t win_len;    // cells of the window
+    int32_t prev_slice; // slice length of the previous row (cells per rank), >= 1
+};
+
+struct ClusterArgs {
+    FwdArgs f;
+    const SliceDesc *slices;  // [L][C]
+    int32_t C;
+    int32_t out_stride;  // floats per `out` buffer
+    int32_t win_stride;  // floats of `win`
+};
+
+template <int MODE, int NT>
+__global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const ClusterArgs cargs)
+{
+    namespace cg = cooperative_groups;
+    constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
+    constexpr int NWARPS = NT / 32;
+    const FwdArgs &args = cargs.f;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int C = cargs.C;
+    const int rank = static_cast<int>(cluster.block_rank());
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *out = reinterpret_cast<float *>(smem_raw);                 // [2][out_stride]
+    float *win = out + 2 * static_cast<size_t>(cargs.out_stride);     // [win_stride]
+    int2 *tap_buf = reinterpret_cast<int2 *>(win + cargs.win_stride);  // [2][K]
+    __shared__ float cl_v[16];
+    __shared__ int cl_t[16];
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int L = args.L, K = args.K;
+    const int64_t n_local = blockIdx.x / C;
+    const int64_t n = args.n_first + n_local;
+    const float *err_n = args.errors + n * L * K;
+    const float INF = pos_inf();
+
+    // Virtual row 0: +0 at t = 0, held in rank 0's first `out` buffer.
+    for (int i = tid; i < 2 * cargs.out_stride; i += NT) out[i] = INF;
+    for (int k = tid; k < K; k += NT) tap_buf[k] = make_int2(args.taps[k].a, __float_as_int(err_n[k]));
+    __syncthreads();
+    if (rank == 0 && tid == 0) out[0] = 0.0f;
+    cluster.sync();
+
+    int prev_width = 1;
+    for (int l = 0; l < L; ++l) {
+        const SliceDesc sd = cargs.slices[l * C + rank];
+        const LayerDesc ld = args.layers[l];
+        const int2 *taps = tap_buf + (l & 1) * K;
+        float *out_prev = out + (l & 1) * cargs.out_stride;
+        float *out_cur = out + ((l + 1) & 1) * cargs.out_stride;
+
+        int2 next_tap = make_int2(0, 0);
+        const bool have_next = (l + 1 < L) && (tid < K);
+        if (have_next)
+            next_tap = make_int2(args.taps[(l + 1) * K + tid].a, __float_as_int(err_n[(l + 1) * K + tid]));
+
+        // Gather the window [q0, q0 + win_len) of the previous row, peer by peer; cells outside
+        // the previous band read as +inf.
+        {
+            const int q_end = sd.q0 + sd.win_len;
+            for (int i = tid; i < sd.win_len; i += NT) {
+                const int q = sd.q0 + i;
+                if (q < 0 || q >= prev_width) win[i] = INF;
+            }
+            const int q_lo = max(sd.q0, 0), q_hi = min(q_end, prev_width);
+            if (q_hi > q_lo) {
+                const int first_rank = q_lo / sd.prev_slice;
+                const int last_rank = (q_hi - 1) / sd.prev_slice;
+                for (int src = first_rank; src <= last_rank; ++src) {
+                    const int seg_lo = max(q_lo, src * sd.prev_slice);
+                    const int seg_hi = min(q_hi, (src + 1) * sd.prev_slice);
+                    const float *remote = (src == rank) ? out_prev : cluster.map_shared_rank(out_prev, src);
+                    const float *from = remote + (seg_lo - src * sd.prev_slice);
+                    float *to = win + (seg_lo - sd.q0);
+                    for (int i = tid; i < seg_hi - seg_lo; i += NT) to[i] = from[i];
+                }
+            }
+        }
+        __syncthreads();
+
+        const float *prev = win - sd.q0;          // prev[q] for q in [q0, q0 + win_len)
+        float *cur = out_cur - sd.slice_lo;       // cur[t_rel] for t_rel in the slice
+        unsigned char *row_base = static_cast<unsigned char *>(args.table) +
+                                  (n_local * args.pitch + ld.rowoff) * (ROWFMT ? 4 : 1);
+        const int MW = (K + 63) >> 6;
+        const unsigned long long *masks = args.span_masks + static_cast<size_t>(sd.mask_off) * MW;
+        const unsigned *kranges = args.span_kranges + sd.mask_off;
+        switch (sd.cpl) {
+#define SPDY_CASE(RR)                                                                             \
+    case RR:                                                                                      \
+        for (int span = warp; span < sd.nspans; span += NWARPS)                                   \
+            process_span<RR, MODE, true>(prev, cur, taps, __ldg(kranges + span),                  \
+                                         masks + span * MW, MW, sd.slice_lo + span * (32 * RR),   \
+                                         lane, row_base, sd.slice_hi);                            \
+        break;
+            SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
+            SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
+            SPDY_CASE(13) SPDY_CASE(14) SPDY_CASE(15) SPDY_CASE(16)
+#undef SPDY_CASE
+            default: break;
+        }
+        if (have_next) tap_buf[((l + 1) & 1) * K + tid] = next_tap;
+        prev_width = ld.width;
+        cluster.sync();  // slices of row l+1 complete everywhere; row l no longer needed
+    }
+
+    // Local minimum over the slice of the last row, then across the cluster through rank 0.
+    const SliceDesc sd = cargs.slices[(L - 1) * C + rank];
+    const LayerDesc ld = args.layers[L - 1];
+    const float *last = out + (L & 1) * cargs.out_stride;
+    float bv = INF;
+    int bt = 0x7fffffff;
+    for (int t = sd.slice_lo + tid; t < sd.slice_hi; t += NT) {
+        const float v = last[t - sd.slice_lo];
+        if (v < bv) {
+            bv = v;
+            bt = t;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+        const int ot = __shfl_xor_sync(0xffffffffu, bt, off);
+        if (ov < bv || (ov == bv && ot < bt)) {
+            bv = ov;
+            bt = ot;
+        }
+    }
+    __shared__ float red_v[32];
+    __shared__ int red_t[32];
+    if (lane == 0) {
+        red_v[warp] = bv;
+        red_t[warp] = bt;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        bv = lane < NWARPS ? red_v[lane] : INF;
+        bt = lane < NWARPS ? red_t[lane] : 0x7fffffff;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+            const int ot = __shfl_xor_sync(0xffffffffu, bt, off);
+            if (ov < bv || (ov == bv && ot < bt)) {
+                bv = ov;
+                bt = ot;
+            }
+        }
+        if (lane == 0) {
+            float *dst_v = cluster.map_shared_rank(cl_v, 0);
+            int *dst_t = cluster.map_shared_rank(cl_t, 0);
+            dst_v[rank] = bv;
+            dst_t[rank] = bt;
+        }
+    }
+    cluster.sync();
+    if (rank == 0 && tid == 0) {
+        bv = cl_v[0];
+        bt = cl_t[0];
+        for (int r = 1; r < C; ++r) {
+            if (cl_v[r] < bv || (cl_v[r] == bv && cl_t[r] < bt)) {
+                bv = cl_v[r];
+                bt = cl_t[r];
+            }
+        }
+        const bool feasible = bv < INF;
+        args.cost[n] = feasible ? bv : INF;
+        args.time_used[n] = feasible ? ld.lo + bt : -1;
     }
 }
 
@@ -567,6 +775,30 @@ const FwdVariant kVariants[] = {
     SPDY_VARIANT(MODE_ROW2, 512, 1),     SPDY_VARIANT(MODE_ROW2, 1024, 1),
 };
 
+using ClusterKernel = void (*)(const ClusterArgs);
+
+struct ClusterVariant {
+    int mode;
+    int threads;
+    ClusterKernel fn;
+};
+
+#define SPDY_CVARIANT(MODE, NT) \
+    ClusterVariant { MODE, NT, spdy_forward_cluster_kernel<MODE, NT> }
+
+const ClusterVariant kClusterVariants[] = {
+    SPDY_CVARIANT(MODE_ARG, 256),  SPDY_CVARIANT(MODE_ARG, 512),  SPDY_CVARIANT(MODE_ARG_PRED, 256),
+    SPDY_CVARIANT(MODE_ARG_PRED, 512), SPDY_CVARIANT(MODE_ROW, 256), SPDY_CVARIANT(MODE_ROW, 512),
+    SPDY_CVARIANT(MODE_ROW2, 256), SPDY_CVARIANT(MODE_ROW2, 512),
+};
+
+const ClusterVariant *find_cluster_variant(int mode, int threads)
+{
+    for (const ClusterVariant &v : kClusterVariants)
+        if (v.mode == mode && v.threads == threads) return &v;
+    return nullptr;
+}
+
 const FwdVariant *find_variant(int mode, int threads)
 {
     for (const FwdVariant &v : kVariants)
@@ -603,6 +835,11 @@ struct spdy_plan {
     std::vector<uint64_t> span_masks;
     std::vector<uint32_t> span_kranges;
     const FwdVariant *variant = nullptr;
+    // cluster variant (cluster > 1)
+    const ClusterVariant *cvariant = nullptr;
+    std::vector<SliceDesc> slices;
+    int32_t out_stride = 0, win_stride = 0;
+    SliceDesc *d_slices = nullptr;
     // device tables (one allocation)
     unsigned char *d_blob = nullptr;
     int32_t *d_times = nullptr;
@@ -744,6 +981,129 @@ int layout_table(spdy_plan *p, int threads, double *efficiency)
     return SPDY_OK;
 }
 
+// Pass shapes when C CTAs share a candidate: every row is cut into C slices of equal length (a
+// multiple of 32 cells); see the cluster kernel for the data flow.
+int layout_cluster(spdy_plan *p, int threads, int C)
+{
+    const int nwarps = threads / 32;
+    const int mw = (p->K + 63) / 64;
+    p->span_masks.clear();
+    p->span_kranges.clear();
+    p->slices.assign(static_cast<size_t>(p->L) * C, SliceDesc{});
+    p->issued_updates = 0;
+    int64_t off = 0, max_slice = 32, max_win = 32, prev_slice = 1;
+    for (int l = 0; l < p->L; ++l) {
+        LayerDesc &ld = p->layers[l];
+        if (off > 0xffffffffLL) return SPDY_ERR_UNSUPPORTED;
+        ld.rowoff = static_cast<uint32_t>(off);
+        ld.cpl = 0;
+        ld.nspans = 0;
+        ld.mask_off = 0;
+        const int64_t width = ld.width;
+        off += round_up(width, 128);
+        const int64_t slice = round_up((width + C - 1) / C, 32);
+        max_slice = std::max(max_slice, slice);
+        int64_t amax = 0;
+        for (int k = 0; k < p->K; ++k) {
+            const TapRange tr = p->taps[static_cast<size_t>(l) * p->K + k];
+            if (tr.b >= tr.a) amax = std::max<int64_t>(amax, tr.a);
+        }
+        for (int r = 0; r < C; ++r) {
+            SliceDesc &sd = p->slices[static_cast<size_t>(l) * C + r];
+            const int64_t lo = std::min<int64_t>(width, r * slice);
+            const int64_t hi = std::min<int64_t>(width, (r + 1) * slice);
+            const int64_t ws = hi - lo;
+            int64_t cpl = 1, nspans = 0;
+            if (ws > 0) {
+                const int64_t per_round = 32LL * nwarps * RMAX;
+                const int64_t rounds = (ws + per_round - 1) / per_round;
+                cpl = (ws + 32LL * nwarps * rounds - 1) / (32LL * nwarps * rounds);
+                cpl = std::min<int64_t>(RMAX, std::max<int64_t>(1, cpl));
+                nspans = (ws + 32 * cpl - 1) / (32 * cpl);
+            }
+            const int64_t span = 32 * cpl;
+            sd.slice_lo = static_cast<int32_t>(lo);
+            sd.slice_hi = static_cast<int32_t>(hi);
+            sd.cpl = static_cast<int32_t>(cpl);
+            sd.nspans = static_cast<int32_t>(nspans);
+            sd.mask_off = static_cast<int32_t>(p->span_masks.size() / mw);
+            sd.q0 = static_cast<int32_t>(lo - amax);
+            sd.win_len = static_cast<int32_t>(nspans > 0 ? amax + nspans * span : 0);
+            sd.prev_slice = static_cast<int32_t>(prev_slice);
+            max_win = std::max<int64_t>(max_win, sd.win_len);
+            for (int64_t sp = 0; sp < nspans; ++sp) {
+                const int64_t s0 = lo + sp * span;
+                uint64_t words[4] = {0, 0, 0, 0};
+                int k_lo = 0, k_hi = 0, count = 0;
+                for (int k = 0; k < p->K; ++k) {
+                    const TapRange tr = p->taps[static_cast<size_t>(l) * p->K + k];
+                    if (tr.b >= tr.a && s0 + span > tr.a && s0 <= tr.b) {
+                        words[k >> 6] |= 1ULL << (k & 63);
+                        p->issued_updates += span;
+                        if (count == 0) k_lo = k;
+                        k_hi = k + 1;
+                        ++count;
+                    }
+                }
+                for (int w = 0; w < mw; ++w) p->span_masks.push_back(words[w]);
+                const uint32_t dense = (count == k_hi - k_lo) ? 1u : 0u;
+                p->span_kranges.push_back(static_cast<uint32_t>(k_lo) | static_cast<uint32_t>(k_hi) << 8 | dense << 16);
+            }
+        }
+        prev_slice = slice;
+    }
+    p->pitch = off;
+    p->out_stride = static_cast<int32_t>(round_up(max_slice, 32));
+    p->win_stride = static_cast<int32_t>(round_up(max_win, 32));
+    p->row_stride = 0;
+    p->smem_bytes = (2LL * p->out_stride + p->win_stride) * 4 + 2LL * p->K * 8;
+    return SPDY_OK;
+}
+
+int choose_cluster_shape(spdy_plan *p, const spdy_options *opts, int64_t smem_per_block)
+{
+    const int requested = (opts && opts->cluster > 1) ? opts->cluster : 0;
+    const int sizes[] = {2, 4, 8};
+    for (int C : sizes) {
+        if (requested && C != requested) continue;
+        for (int threads : {512, 256}) {
+            if (opts && opts->threads && opts->threads != threads) continue;
+            if (threads < p->K) continue;
+            int rc = layout_cluster(p, threads, C);
+            if (rc != SPDY_OK) return rc;
+            if (p->smem_bytes > smem_per_block) continue;
+            // Narrow slices do not fill 16 warps; prefer the smaller CTA then.
+            if (threads == 512 && !(opts && opts->threads) && p->out_stride < 32 * 16 * 4) continue;
+            p->cluster = C;
+            p->threads = threads;
+            p->cvariant = find_cluster_variant(p->mode, threads);
+            if (!p->cvariant) return SPDY_ERR_INVALID_ARG;
+            p->ctas_per_sm = 1;
+            if (p->device >= 0) {
+                SPDY_CUDA_TRY(cudaFuncSetAttribute(p->cvariant->fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   static_cast<int>(p->smem_bytes)));
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(static_cast<unsigned>(C), 1, 1);
+                cfg.blockDim = dim3(static_cast<unsigned>(threads), 1, 1);
+                cfg.dynamicSmemBytes = static_cast<size_t>(p->smem_bytes);
+                cudaLaunchAttribute attr;
+                attr.id = cudaLaunchAttributeClusterDimension;
+                attr.val.clusterDim.x = static_cast<unsigned>(C);
+                attr.val.clusterDim.y = 1;
+                attr.val.clusterDim.z = 1;
+                cfg.attrs = &attr;
+                cfg.numAttrs = 1;
+                int clusters = 0;
+                SPDY_CUDA_TRY(cudaOccupancyMaxActiveClusters(&clusters, p->cvariant->fn, &cfg));
+                if (clusters < 1) continue;
+                p->ctas_per_sm = std::max(1, clusters * C / std::max(1, p->sm_count));
+            }
+            return SPDY_OK;
+        }
+    }
+    return requested ? SPDY_ERR_INVALID_ARG : SPDY_ERR_UNSUPPORTED;
+}
+
 int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
 {
     int64_t smem_per_sm = 233472, smem_per_block = 232448;
@@ -768,8 +1128,11 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
         if (!(row_mode || arg_mode)) return SPDY_ERR_INVALID_ARG;
         if (row_mode != (p->table_format == SPDY_TABLE_ROW_F32)) return SPDY_ERR_INVALID_ARG;
     }
-    p->cluster = (opts && opts->cluster) ? opts->cluster : 1;
-    if (p->cluster != 1) return SPDY_ERR_UNSUPPORTED;
+    p->cluster = 1;
+    if (opts && opts->cluster != 0 && opts->cluster != 1 && opts->cluster != 2 && opts->cluster != 4 &&
+        opts->cluster != 8)
+        return SPDY_ERR_INVALID_ARG;
+    if (opts && opts->cluster > 1) return choose_cluster_shape(p, opts, smem_per_block);
 
     // Candidate CTA sizes; keep the one whose rounds are fullest, preferring more resident warps.
     const int sizes[] = {128, 256, 512, 1024};
@@ -792,7 +1155,12 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
             best_threads = threads;
         }
     }
-    if (best_threads == 0) return (opts && opts->threads) ? SPDY_ERR_INVALID_ARG : SPDY_ERR_UNSUPPORTED;
+    if (best_threads == 0) {
+        // No single CTA can hold two rows of this width: split each candidate over a cluster,
+        // unless the caller insisted on one CTA.
+        if (opts && opts->cluster == 1) return SPDY_ERR_UNSUPPORTED;
+        return choose_cluster_shape(p, opts, smem_per_block);
+    }
     int rc = layout_table(p, best_threads, nullptr);
     if (rc != SPDY_OK) return rc;
     p->threads = best_threads;
@@ -820,8 +1188,11 @@ int upload_tables(spdy_plan *p)
     const size_t off_masks = off_taps + round_up(n_times * sizeof(TapRange), 256);
     const size_t off_kranges = off_masks + round_up(p->span_masks.size() * sizeof(uint64_t) + 8, 256);
     const size_t off_status = off_kranges + round_up(p->span_kranges.size() * sizeof(uint32_t) + 4, 256);
-    const size_t total = off_status + 256;
+    const size_t off_slices = off_status + 256;
+    const size_t total = off_slices + round_up(p->slices.size() * sizeof(SliceDesc) + 32, 256);
     std::vector<unsigned char> host(total, 0);
+    if (!p->slices.empty())
+        std::memcpy(host.data() + off_slices, p->slices.data(), p->slices.size() * sizeof(SliceDesc));
     std::memcpy(host.data(), p->times.data(), n_times * sizeof(int32_t));
     std::memcpy(host.data() + off_layers, p->layers.data(), p->L * sizeof(LayerDesc));
     std::memcpy(host.data() + off_taps, p->taps.data(), n_times * sizeof(TapRange));
@@ -842,6 +1213,7 @@ int upload_tables(spdy_plan *p)
     p->d_masks = reinterpret_cast<unsigned long long *>(p->d_blob + off_masks);
     p->d_kranges = reinterpret_cast<unsigned *>(p->d_blob + off_kranges);
     p->d_status = reinterpret_cast<int32_t *>(p->d_blob + off_status);
+    p->d_slices = reinterpret_cast<SliceDesc *>(p->d_blob + off_slices);
     return SPDY_OK;
 }
 
@@ -1033,7 +1405,29 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
         fa.K = plan->K;
         fa.row_stride = plan->row_stride;
         // Grid x is limited to 2^31-1 CTAs, far above any wave that fits in memory.
-        plan->variant->fn<<<static_cast<unsigned>(count), plan->threads, static_cast<size_t>(plan->smem_bytes), stream>>>(fa);
+        if (plan->cluster > 1) {
+            ClusterArgs ca;
+            ca.f = fa;
+            ca.slices = plan->d_slices;
+            ca.C = plan->cluster;
+            ca.out_stride = plan->out_stride;
+            ca.win_stride = plan->win_stride;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(static_cast<unsigned>(count * plan->cluster), 1, 1);
+            cfg.blockDim = dim3(static_cast<unsigned>(plan->threads), 1, 1);
+            cfg.dynamicSmemBytes = static_cast<size_t>(plan->smem_bytes);
+            cfg.stream = stream;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = static_cast<unsigned>(plan->cluster);
+            attr.val.clusterDim.y = 1;
+            attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            SPDY_CUDA_TRY(cudaLaunchKernelEx(&cfg, plan->cvariant->fn, ca));
+        } else {
+            plan->variant->fn<<<static_cast<unsigned>(count), plan->threads, static_cast<size_t>(plan->smem_bytes), stream>>>(fa);
+        }
         SPDY_CUDA_TRY(cudaGetLastError());
         if (ev) SPDY_CUDA_TRY(cudaEventRecord(ev[1], stream));
 

@@ -196,3 +196,41 @@ def test_full_size_bert_base_batch_in_the_benchmark_configuration():
     assert_same((p[sample], c[sample], t[sample]), ref)
     for n in sample[:4]:
         check_solution(wl.errors[n], wl.times, wl.B, p[n], c[n], int(t[n]))
+
+
+@pytest.mark.parametrize("cluster", [2, 4, 8])
+@pytest.mark.parametrize("mode", [1, 2, 3, 4])
+def test_cluster_split_of_one_candidate_gives_the_same_answer(cluster, mode):
+    """A candidate cut over a thread-block cluster (slices of every row, windows gathered through
+    distributed shared memory) must match the oracle like the single-CTA kernel."""
+    fmt = 1 if mode in (1, 2) else 2
+    wl = W.make_workload(2, N=6)
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+    assert_same(gpu_solve(wl, fmt, cluster=cluster, forward_mode=mode), ref)
+    for seed in (10_003, 10_007, 21, 33):  # rows narrower than the cluster: empty slices
+        tiny = W.tiny_random_instance(seed, exact=seed >= 10_000, N=3)
+        assert_same(gpu_solve(tiny, fmt, cluster=cluster, forward_mode=mode),
+                    oracle.solve_batch(tiny.errors, tiny.times, tiny.B))
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_budget_100000_needs_a_cluster(fmt):
+    """B = 100000: a band-limited row is about 210 KB, so two rows cannot live in one CTA."""
+    wl = W.make_workload(4, N=5, B=100000)
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+    assert plan.info["cluster"] > 1
+    plan.close()
+    assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+
+
+def test_cluster_with_ties_and_wide_rows():
+    rng = np.random.default_rng(78)
+    L, K, B, N = 10, 7, 5000, 12
+    times = rng.integers(0, 900, size=(L, K)).astype(np.int32)
+    times[3, :] = 0
+    errors = rng.choice(np.array([0, 0.25, 0.5, 1.0], np.float32), size=(N, L, K)).astype(np.float32)
+    wl = W.Workload("ties-cluster", times, errors, B)
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+    for cluster in (2, 4, 8):
+        for fmt in FORMATS:
+            assert_same(gpu_solve(wl, fmt, cluster=cluster), ref)

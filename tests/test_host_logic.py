@@ -130,3 +130,18 @@ def test_infeasible_and_degenerate_plans():
     assert info["feasible"] == 1 and info["max_width"] == 1
     over = np.array([[50, 60]], np.int32)  # every choice above the budget
     assert binding.Plan(over, 10, device=-1).info["feasible"] == 0
+
+
+def test_wide_rows_choose_a_cluster():
+    wl = W.make_workload(4, N=1, B=100000)
+    info = binding.Plan(wl.times, wl.B, device=-1).info
+    assert info["cluster"] in (2, 4, 8) and info["smem_bytes"] <= 232448
+    with pytest.raises(binding.SpdyError) as e:  # one CTA cannot hold it
+        binding.Plan(wl.times, wl.B, device=-1, cluster=1)
+    assert e.value.status == -3
+    with pytest.raises(binding.SpdyError):
+        binding.Plan(wl.times, wl.B, device=-1, cluster=3)
+    small = W.make_workload(2, N=1)
+    for c in (2, 4, 8):
+        info = binding.Plan(small.times, small.B, device=-1, cluster=c).info
+        assert info["cluster"] == c and info["useful_updates"] <= info["issued_updates"]
