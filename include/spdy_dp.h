@@ -44,7 +44,8 @@ typedef enum spdy_status {
     SPDY_ERR_UNSUPPORTED = -3,        /* rows too wide for the largest launch shape on this device */
     SPDY_ERR_CUDA = -4,               /* a CUDA runtime call failed; see spdy_last_cuda_error() */
     SPDY_ERR_NO_MEMORY = -5,          /* host or device allocation failed */
-    SPDY_ERR_INTERNAL = -6            /* a self-check inside the kernels failed */
+    SPDY_ERR_INTERNAL = -6,           /* a self-check inside the kernels failed */
+    SPDY_ERR_STATIC_LIMIT = -7        /* spdy_solve_batch_static: problem exceeds its built-in scratch */
 } spdy_status;
 
 /*
@@ -176,6 +177,43 @@ int spdy_plan_check_status(spdy_plan *plan, void *cuda_stream);
  */
 int spdy_plan_enable_timing(spdy_plan *plan, int on);
 int spdy_plan_last_timing(spdy_plan *plan, float *forward_ms_host, float *walkback_ms_host);
+
+/*
+ * (No counterpart in the paper: a deployment convenience.)
+ *
+ * The same path - forward dynamic program, final minimum, walk back - for callers that are not
+ * allowed to allocate device memory: code that runs under a framework which owns the whole
+ * device heap and forbids side allocations, services that fix their memory footprint at start-up,
+ * or a process that has already handed every free byte to another pool.  This call makes no CUDA
+ * allocation of any kind (no cudaMalloc / cudaFree / pool or async allocation, no allocating
+ * library routine); its only scratch is an array of SPDY_STATIC_SCRATCH_BYTES compiled into the
+ * library, which every device that loads the library holds until the process exits.  The array
+ * carries the plan's small tables and the walk-back table (one byte per live cell); a batch whose
+ * table is larger runs as several waves.  The caller still passes every input and output.
+ *
+ *   errors_dev     device, [N][L][K] fp32.          times_host  host, [L][K] int32.
+ *   profile_dev / cost_dev / time_used_dev          device outputs as for spdy_solve_batch.
+ *
+ * Behaviour to know about:
+ *   - Works on the current device.  Synchronous: waits for `cuda_stream` before returning.
+ *   - The first call on each device looks up the array's device address through the runtime
+ *     (which may load the module); make that first call outside any stream capture.
+ *   - All calls on one device share the one array, and it keeps whatever the last call left.  The
+ *     only word that must start at zero, the self-check flag, is cleared on the stream at each
+ *     call.  Two calls whose GPU work overlaps (different streams or host threads) race on the
+ *     array: serialise them.
+ *   - Limits: returns SPDY_ERR_STATIC_LIMIT when the plan tables plus ONE candidate's table do
+ *     not fit the array, or when a row is too wide for a single CTA (the cluster variant is not
+ *     offered here).  The BERT-base shape (L 72, K 42, B 10000) needs about 0.4 MB per candidate.
+ * Other errors as for spdy_solve_batch (INVALID_ARG, CUDA, INTERNAL).
+ */
+#define SPDY_STATIC_SCRATCH_BYTES (64u << 20)
+int spdy_solve_batch_static(const float *errors_dev, const int32_t *times_host, int64_t N, int32_t L,
+                            int32_t K, int32_t B, uint8_t *profile_dev, float *cost_dev,
+                            int32_t *time_used_dev, void *cuda_stream);
+
+/* Size in bytes of the array spdy_solve_batch_static works in (SPDY_STATIC_SCRATCH_BYTES). */
+size_t spdy_static_scratch_bytes(void);
 
 /* Static, human-readable text for a status code. */
 const char *spdy_strerror(int status);

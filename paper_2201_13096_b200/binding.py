@@ -20,7 +20,8 @@ SPDY_TABLE_DEFAULT, SPDY_TABLE_ARG_U8, SPDY_TABLE_ROW_F32 = 0, 1, 2
 EXPORTS = (
     "spdy_plan_create", "spdy_plan_destroy", "spdy_plan_get_info", "spdy_plan_get_bands",
     "spdy_workspace_bytes", "spdy_solve_batch", "spdy_solve_batch_host", "spdy_solve_batch_simple",
-    "spdy_plan_check_status", "spdy_plan_enable_timing", "spdy_plan_last_timing", "spdy_strerror", "spdy_last_cuda_error", "spdy_version",
+    "spdy_plan_check_status", "spdy_plan_enable_timing", "spdy_plan_last_timing",
+    "spdy_solve_batch_static", "spdy_static_scratch_bytes", "spdy_strerror", "spdy_last_cuda_error", "spdy_version",
 )
 
 
@@ -90,6 +91,9 @@ def _load():
     lib.spdy_plan_last_timing.restype = ctypes.c_int
     lib.spdy_plan_last_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
                                           ctypes.POINTER(ctypes.c_float)]
+    lib.spdy_solve_batch_static.restype = ctypes.c_int
+    lib.spdy_solve_batch_static.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
+    lib.spdy_static_scratch_bytes.restype = ctypes.c_size_t
     lib.spdy_strerror.restype = ctypes.c_char_p
     lib.spdy_strerror.argtypes = [ctypes.c_int]
     lib.spdy_last_cuda_error.restype = ctypes.c_int
@@ -239,4 +243,31 @@ def solve_batch_simple(errors, times, B: int, stream=None):
                                            profile.data_ptr(), cost.data_ptr(),
                                            time_used.data_ptr(), _stream_handle(stream)),
            "spdy_solve_batch_simple")
+    return profile, cost, time_used
+
+
+def solve_batch_static(errors, times, B: int, profile=None, cost=None, time_used=None, stream=None):
+    """``spdy_solve_batch_static``: the whole path without any device allocation by the library.
+    For callers that may not allocate on the device (a framework owns the heap, or the memory
+    budget is fixed at start-up): the library works inside an array compiled into it.  ``errors``
+    is a CUDA fp32 tensor [N][L][K], ``times`` a host int32 array [L][K]; pass the three output
+    tensors to keep this wrapper from allocating them with torch.  Synchronous.  Calls must not
+    overlap on one device, and the first call per device must come before any stream capture."""
+    import torch
+
+    t = np.ascontiguousarray(np.asarray(times), dtype=np.int32)
+    N, L, K = (int(x) for x in errors.shape)
+    if t.shape != (L, K):
+        raise ValueError("times must be [L][K] matching errors")
+    dev = errors.device
+    if profile is None:
+        profile = torch.empty((N, L), dtype=torch.uint8, device=dev)
+    if cost is None:
+        cost = torch.empty(N, dtype=torch.float32, device=dev)
+    if time_used is None:
+        time_used = torch.empty(N, dtype=torch.int32, device=dev)
+    _check(_load().spdy_solve_batch_static(errors.data_ptr(), t.ctypes.data_as(ctypes.c_void_p), N, L,
+                                           K, int(B), profile.data_ptr(), cost.data_ptr(),
+                                           time_used.data_ptr(), _stream_handle(stream)),
+           "spdy_solve_batch_static")
     return profile, cost, time_used

@@ -16,6 +16,7 @@
 #include <algorithm>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -1253,6 +1254,7 @@ const char *spdy_strerror(int status)
         case SPDY_ERR_CUDA: return "CUDA runtime call failed";
         case SPDY_ERR_NO_MEMORY: return "out of memory";
         case SPDY_ERR_INTERNAL: return "internal self-check failed";
+        case SPDY_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of spdy_solve_batch_static";
         default: return "unknown status";
     }
 }
@@ -1602,6 +1604,141 @@ int spdy_solve_batch_simple(const float *errors_dev, const int32_t *times_dev, i
     if (rc == SPDY_OK) rc = spdy_plan_check_status(plan, stream);
     if (ws) cudaFree(ws);
     spdy_plan_destroy(plan);
+    return rc;
+}
+
+// ----------------------------------------------------------------------------------------------
+// Entry point that performs no device allocation
+// ----------------------------------------------------------------------------------------------
+
+}  // extern "C"
+
+namespace {
+
+// Built-in scratch of spdy_solve_batch_static: the plan's small tables at the front, the
+// walk-back table behind them.  Resident on every device that loads this library, until exit.
+constexpr size_t kStaticScratchBytes = SPDY_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char *g_static_base[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device.  In host code the array's name is
+// only a handle, never a pointer a kernel may use; the address comes from the runtime, once per
+// device.
+int static_scratch_address(int device, unsigned char **out)
+{
+    if (device < 0 || device >= kMaxDevices) return SPDY_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_base[device]) {
+        void *ptr = nullptr;
+        SPDY_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        if (!ptr) return SPDY_ERR_CUDA;
+        g_static_base[device] = static_cast<unsigned char *>(ptr);
+    }
+    *out = g_static_base[device];
+    return SPDY_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t spdy_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+int spdy_solve_batch_static(const float *errors_dev, const int32_t *times_host, int64_t N, int32_t L,
+                            int32_t K, int32_t B, uint8_t *profile_dev, float *cost_dev,
+                            int32_t *time_used_dev, void *cuda_stream)
+{
+    if (!times_host || L < 1 || K < 1 || K > 255 || B < 0 || N < 0) return SPDY_ERR_INVALID_ARG;
+    if (N == 0) return SPDY_OK;
+    if (!errors_dev || !profile_dev || !cost_dev || !time_used_dev) return SPDY_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int device = 0;
+    SPDY_CUDA_TRY(cudaGetDevice(&device));
+    unsigned char *base = nullptr;
+    int rc = static_scratch_address(device, &base);
+    if (rc != SPDY_OK) return rc;
+
+    // Host-side plan (bands, pass shapes) with the one-byte table so more candidates fit a wave.
+    spdy_plan *p = new (std::nothrow) spdy_plan();
+    if (!p) return SPDY_ERR_NO_MEMORY;
+    p->L = L;
+    p->K = K;
+    p->B = B;
+    p->device = device;
+    spdy_options opts = {};
+    opts.table_format = SPDY_TABLE_ARG_U8;
+    opts.cluster = 1;  // the cluster variant's wider rows would not leave room for a table anyway
+    try {
+        p->times.assign(times_host, times_host + static_cast<size_t>(L) * K);
+        rc = build_bands(p);
+        if (rc == SPDY_OK) rc = choose_launch_shape(p, &opts);
+    } catch (const std::bad_alloc &) {
+        rc = SPDY_ERR_NO_MEMORY;
+    }
+    if (rc == SPDY_ERR_UNSUPPORTED) rc = SPDY_ERR_STATIC_LIMIT;
+    if (rc != SPDY_OK) {
+        spdy_plan_destroy(p);
+        return rc;
+    }
+
+    // Carve the plan tables out of the front of the scratch.
+    const size_t n_times = static_cast<size_t>(L) * K;
+    const size_t off_layers = round_up(n_times * sizeof(int32_t), 256);
+    const size_t off_taps = off_layers + round_up(L * sizeof(LayerDesc), 256);
+    const size_t off_masks = off_taps + round_up(n_times * sizeof(TapRange), 256);
+    const size_t off_kranges = off_masks + round_up(p->span_masks.size() * sizeof(uint64_t) + 8, 256);
+    const size_t off_status = off_kranges + round_up(p->span_kranges.size() * sizeof(uint32_t) + 4, 256);
+    const size_t off_table = off_status + 256;
+    const size_t one = p->feasible ? spdy_workspace_bytes(p, 1) : 0;
+    if (off_table + one > kStaticScratchBytes) {
+        spdy_plan_destroy(p);
+        return SPDY_ERR_STATIC_LIMIT;
+    }
+    p->d_times = reinterpret_cast<int32_t *>(base);
+    p->d_layers = reinterpret_cast<LayerDesc *>(base + off_layers);
+    p->d_taps = reinterpret_cast<TapRange *>(base + off_taps);
+    p->d_masks = reinterpret_cast<unsigned long long *>(base + off_masks);
+    p->d_kranges = reinterpret_cast<unsigned *>(base + off_kranges);
+    p->d_status = reinterpret_cast<int32_t *>(base + off_status);
+    cudaError_t err = cudaSuccess;
+    auto copy = [&](void *dst, const void *src, size_t bytes) {
+        if (err == cudaSuccess && bytes > 0) err = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, stream);
+    };
+    copy(p->d_times, p->times.data(), n_times * sizeof(int32_t));
+    copy(p->d_layers, p->layers.data(), L * sizeof(LayerDesc));
+    copy(p->d_taps, p->taps.data(), n_times * sizeof(TapRange));
+    copy(p->d_masks, p->span_masks.data(), p->span_masks.size() * sizeof(uint64_t));
+    copy(p->d_kranges, p->span_kranges.data(), p->span_kranges.size() * sizeof(uint32_t));
+    // The array keeps the previous call's contents; only the self-check word must start at zero.
+    if (err == cudaSuccess) err = cudaMemsetAsync(p->d_status, 0, 256, stream);
+    if (err != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(err);
+        cudaStreamSynchronize(stream);
+        spdy_plan_destroy(p);
+        return SPDY_ERR_CUDA;
+    }
+    const size_t table_bytes = p->feasible ? (kStaticScratchBytes - off_table) / one * one : 0;
+    rc = spdy_solve_batch(p, errors_dev, N, profile_dev, cost_dev, time_used_dev, base + off_table,
+                          table_bytes, stream);
+    int32_t word = 0;
+    if (rc == SPDY_OK) {
+        err = cudaMemcpyAsync(&word, p->d_status, sizeof(word), cudaMemcpyDeviceToHost, stream);
+        if (err != cudaSuccess) {
+            g_last_cuda_error = static_cast<int>(err);
+            rc = SPDY_ERR_CUDA;
+        }
+    }
+    // The host tables above must outlive the copies, so wait before releasing them.
+    err = cudaStreamSynchronize(stream);
+    if (rc == SPDY_OK && err != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(err);
+        rc = SPDY_ERR_CUDA;
+    }
+    if (rc == SPDY_OK && word != 0) rc = SPDY_ERR_INTERNAL;
+    spdy_plan_destroy(p);  // frees host tables only: this plan owns no device memory
     return rc;
 }
 
