@@ -184,7 +184,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
 
-    from paper_2201_13096_b200 import binding, workloads as W
+    from paper_2201_13096_b200 import binding, sharding, workloads as W
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -201,7 +201,8 @@ def run_ours(args):
     # stream against the same timing table; no data-path collective.
     probe = W.make_workload(args.config, N=1, B=args.budget)
     n_per_rank = args.n if args.n is not None else {1: 1024, 2: 4096, 3: 1024, 4: 4096}[args.config]
-    wl = W.make_workload(args.config, N=n_per_rank, B=args.budget, start=rank * n_per_rank)
+    start, count = sharding.shard_range(world * n_per_rank, rank, world)
+    wl = W.make_workload(args.config, N=count, B=args.budget, start=start)
     assert np.array_equal(probe.times, wl.times)
     fmt = {"default": 0, "arg": 1, "row": 2}[args.table]
     if args.mode:
@@ -251,10 +252,7 @@ def run_ours(args):
         barrier()
     step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
     total_ms = float(sum(step_ms))
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = sharding.max_over_ranks(total_ms, dev)
     plan.check_status()
 
     # End to end through the host-buffer entry point: pinned host inputs, copies inside the timing.
@@ -272,15 +270,12 @@ def run_ours(args):
             binding.solve_batch_host(plan, h_err, h_prof, h_cost, h_time, stream)
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = sharding.max_over_ranks(e2e_s, dev)
         same = (torch.equal(h_prof, profile.cpu()) and torch.equal(h_time, time_used.cpu())
                 and h_cost.numpy().tobytes() == cost.cpu().numpy().tobytes())
         if not same:
             raise SystemExit("host-buffer path disagrees with the device-buffer path")
-        e2e = {"value": world * wl.N * args.steps / e2e_s, "unit": "candidates/s",
+        e2e = {"value": sharding.whole_job_rate(wl.N * args.steps, world, e2e_s), "unit": "candidates/s",
                "h2d_bytes_per_step": int(h_err.numel() * 4),
                "d2h_bytes_per_step": int(wl.N * (wl.L + 8)), "ms_per_step": 1e3 * e2e_s / args.steps}
 
@@ -290,7 +285,7 @@ def run_ours(args):
         return
 
     ms_per_step = total_ms / args.steps
-    cand_per_s = world * wl.N / (ms_per_step * 1e-3)
+    cand_per_s = sharding.whole_job_rate(wl.N, world, ms_per_step * 1e-3)
     fwd = float(np.mean(fwd_ms))
     back = float(np.mean(back_ms))
     peaks = {}
