@@ -28,6 +28,12 @@ SM_COUNT_NOMINAL = 148
 SM_MAX_MHZ_NOMINAL = 1965.0
 CELLS_PER_CLK_PER_SM = 32.0  # one 4-byte shared-memory read per cell update, 32 banks x 4 B per clock
 
+# DRAM bytes (read + write) of the forward kernel per candidate from an ncu capture of one wave
+# (592 candidates) of the BERT-base shape; traffic grows in proportion to N.  Valid only for the
+# library version the counters were taken with.
+NCU_TRAFFIC = {"version": 1001, "workload_prefix": "bert-base-L72-K42-B10000",
+               "bytes_per_candidate": {"row_f32": 764.2e6 / 592, "arg_u8": 157.0e6 / 592}}
+
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -300,6 +306,11 @@ def run_ours(args):
     hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
     cellb = 4 if info["table_format"] == 2 else 1
     hbm_bytes = wl.N * (info["band_cells"] * cellb + wl.L * wl.K * 4)
+    table_name = {1: "arg_u8", 2: "row_f32"}[info["table_format"]]
+    traffic = None
+    if (binding.library().spdy_version() == NCU_TRAFFIC["version"] and info["cluster"] == 1
+            and wl.name.startswith(NCU_TRAFFIC["workload_prefix"]) and wl.B == 10000):
+        traffic = NCU_TRAFFIC["bytes_per_candidate"][table_name] * wl.N / waves
     line = {
         "metric": "candidate_profiles_per_s", "value": cand_per_s, "unit": "candidates/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
@@ -309,7 +320,7 @@ def run_ours(args):
                    "l2": "256 MiB buffer rewritten between timed steps (L2 flush); the walk-back table "
                          f"written per step is {info['table_bytes_per_candidate'] * wl.N / 1e6:.0f} MB",
                    "timing": "sum of per-step CUDA-event pairs on the launch stream, max over ranks",
-                   "table_format": {1: "arg_u8", 2: "row_f32"}[info["table_format"]],
+                   "table_format": table_name,
                    "threads": info["threads"], "ctas_per_sm": info["ctas_per_sm"], "span": info["span"],
                    "cluster": info["cluster"],
                    "waves": int(waves)},
@@ -318,7 +329,8 @@ def run_ours(args):
         "roofline": {
             "bound": "alu", "kernel": "spdy_forward_kernel",
             "achieved": achieved / 1e9, "peak": peak_cells / 1e9, "unit": "Gcell-updates/s",
-            "frac": achieved / peak_cells, "traffic": None,
+            "frac": achieved / peak_cells, "traffic": traffic,
+            "traffic_unit": "bytes per launch (ncu dram read+write on one wave, scaled by N)",
             "peak_is": f"{info['sm_count']} SMs x {sm_max:.0f} MHz x 32 four-byte shared-memory reads per clock "
                        "(one read per cell update); of nominal unit counts, max clock of measured",
             "kernel_ms": fwd, "walkback_ms": back,

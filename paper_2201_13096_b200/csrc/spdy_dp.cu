@@ -1240,7 +1240,7 @@ struct DeviceGuard {
 
 extern "C" {
 
-int spdy_version(void) { return 1000; }
+int spdy_version(void) { return 1001; }
 
 int spdy_last_cuda_error(void) { return g_last_cuda_error; }
 
