@@ -92,6 +92,9 @@ typedef struct spdy_plan_info {
     int64_t useful_updates; /* sum over (layer, choice) of cells whose source lies in the previous band */
     int64_t issued_updates; /* cell updates the kernel actually issues per candidate (span granularity) */
     int64_t nominal_updates;/* L*K*B per candidate, the unit of the headline metric */
+    int64_t distinct_updates; /* like useful_updates after choices of a layer with equal times are merged
+                                 into one shift (row-value table only; equals useful_updates otherwise):
+                                 the cell updates the forward pass has to perform */
 } spdy_plan_info;
 
 typedef struct spdy_plan spdy_plan; /* opaque; owns only its own small host and device tables */

@@ -59,11 +59,19 @@ struct LayerDesc {
     int32_t cpl;     // cells per lane per pass, 1..RMAX
     int32_t nspans;  // passes needed to cover the band: ceil(width / (32*cpl))
     int32_t mask_off;  // index of the layer's first pass in the pass-mask table
-    int32_t pad1;
+    int32_t nslots;    // shift slots of the layer (see TapRange)
 };
 
 // One (layer, choice) pair in band coordinates: the choice contributes to cells t_rel in [a, b]
 // and reads the previous row at t_rel - a.  An unusable choice has b < a.
+//
+// The kernels walk "shift slots" rather than choices.  With a byte table (the winning choice is
+// stored) slot u of a layer is choice u.  With a row-value table only the minimum matters, and
+// since x -> fl32(x + e) is non-decreasing in e, the choices of a layer that share one time
+// collapse exactly into one slot carrying the smallest of their errors:
+//   min_k fl32(D[t - tau] + e_k) == fl32(D[t - tau] + min_k e_k)   over the k with times[l][k] == tau.
+// Slots are then the distinct usable times in ascending order; slot_ptr/slot_member list the
+// choices behind each slot.  (D never holds -0, so which zero the minimum picks does not matter.)
 struct TapRange {
     int32_t a;
     int32_t b;
@@ -71,10 +79,12 @@ struct TapRange {
 
 struct FwdArgs {
     const float *errors;      // [N][L][K]
-    const TapRange *taps;     // [L][K]
+    const TapRange *slots;    // [L][K], the first layers[l].nslots of a layer are valid
+    const uint8_t *slot_ptr;     // [L][K+1]: members of slot u are slot_member[slot_ptr[u] .. slot_ptr[u+1])
+    const uint8_t *slot_member;  // [L][K]: choice indices grouped by slot
     const LayerDesc *layers;  // [L]
-    const unsigned long long *span_masks;  // per pass: one bit per choice that overlaps it
-    const unsigned *span_kranges;          // per pass: k_lo | k_hi << 8 | dense << 16
+    const unsigned long long *span_masks;  // per pass: one bit per slot that overlaps it
+    const unsigned *span_kranges;          // per pass: u_lo | u_hi << 8 | dense << 16
     void *table;              // wave-local walk-back table
     float *cost;              // [N]
     int32_t *time_used;       // [N]
@@ -85,6 +95,20 @@ struct FwdArgs {
 };
 
 __device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
+
+// (shift, error bits) of slot u of layer l for one candidate: the smallest error among the
+// slot's choices (a single choice unless equal times were merged).
+__device__ __forceinline__ int2 stage_slot(const FwdArgs &args, const float *err_n, const int l, const int u)
+{
+    const int K = args.K;
+    const uint8_t *ptr = args.slot_ptr + static_cast<size_t>(l) * (K + 1);
+    const uint8_t *member = args.slot_member + static_cast<size_t>(l) * K;
+    const float *err_l = err_n + static_cast<size_t>(l) * K;
+    const int j0 = ptr[u], j1 = ptr[u + 1];
+    float e = err_l[member[j0]];
+    for (int j = j0 + 1; j < j1; ++j) e = fminf(e, err_l[member[j]]);
+    return make_int2(args.slots[static_cast<size_t>(l) * K + u].a, __float_as_int(e));
+}
 
 // Two independent round-to-nearest fp32 adds in one instruction: (x, y) += (e, e).
 __device__ __forceinline__ void add2_rn(float &x, float &y, unsigned long long e2)
@@ -330,7 +354,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
 
     // Both buffers start as +inf everywhere; D_0 is +0 at t = 0 (Eq. 3 via a virtual row 0).
     for (int i = tid; i < 2 * args.row_stride; i += NT) rows[i] = INF;
-    for (int k = tid; k < K; k += NT) tap_buf[k] = make_int2(args.taps[k].a, __float_as_int(err_n[k]));
+    for (int u = tid; u < args.layers[0].nslots; u += NT) tap_buf[u] = stage_slot(args, err_n, 0, u);
     __syncthreads();
     if (tid == 0) rows[PAD] = 0.0f;
     __syncthreads();
@@ -341,12 +365,11 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         const int2 *taps = tap_buf + (l & 1) * K;
         const LayerDesc ld = args.layers[l];
 
-        // Fetch the next layer's choices early; they are parked in shared memory after the pass.
-        // (NT >= K is guaranteed by the host, so one thread per choice suffices.)
+        // Fetch the next layer's slots early; they are parked in shared memory after the pass.
+        // (NT >= K is guaranteed by the host, so one thread per slot suffices.)
         int2 next_tap = make_int2(0, 0);
-        const bool have_next = (l + 1 < L) && (tid < K);
-        if (have_next)
-            next_tap = make_int2(args.taps[(l + 1) * K + tid].a, __float_as_int(err_n[(l + 1) * K + tid]));
+        const bool have_next = (l + 1 < L) && (tid < args.layers[l + 1].nslots);
+        if (have_next) next_tap = stage_slot(args, err_n, l + 1, tid);
 
         unsigned char *row_base = static_cast<unsigned char *>(args.table) +
                                   (n_local * args.pitch + ld.rowoff) * (ROWFMT ? 4 : 1);
@@ -487,7 +510,7 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
 
     // Virtual row 0: +0 at t = 0, held in rank 0's first `out` buffer.
     for (int i = tid; i < 2 * cargs.out_stride; i += NT) out[i] = INF;
-    for (int k = tid; k < K; k += NT) tap_buf[k] = make_int2(args.taps[k].a, __float_as_int(err_n[k]));
+    for (int u = tid; u < args.layers[0].nslots; u += NT) tap_buf[u] = stage_slot(args, err_n, 0, u);
     __syncthreads();
     if (rank == 0 && tid == 0) out[0] = 0.0f;
     cluster.sync();
@@ -501,9 +524,8 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
         float *out_cur = out + ((l + 1) & 1) * cargs.out_stride;
 
         int2 next_tap = make_int2(0, 0);
-        const bool have_next = (l + 1 < L) && (tid < K);
-        if (have_next)
-            next_tap = make_int2(args.taps[(l + 1) * K + tid].a, __float_as_int(err_n[(l + 1) * K + tid]));
+        const bool have_next = (l + 1 < L) && (tid < args.layers[l + 1].nslots);
+        if (have_next) next_tap = stage_slot(args, err_n, l + 1, tid);
 
         // Gather the window [q0, q0 + win_len) of the previous row, peer by peer; cells outside
         // the previous band read as +inf.
@@ -828,11 +850,14 @@ struct spdy_plan {
     int64_t smem_bytes = 0;
     int32_t row_stride = 0;
     int64_t pitch = 0;  // table cells per candidate
-    int64_t band_cells = 0, useful_updates = 0, issued_updates = 0;
+    int64_t band_cells = 0, useful_updates = 0, distinct_updates = 0, issued_updates = 0;
     int32_t max_width = 0;
     std::vector<int32_t> times;
     std::vector<LayerDesc> layers;
-    std::vector<TapRange> taps;
+    std::vector<TapRange> taps;       // [L][K] by choice
+    std::vector<TapRange> slots;      // [L][K] by shift slot (first layers[l].nslots valid)
+    std::vector<uint8_t> slot_ptr;    // [L][K+1]
+    std::vector<uint8_t> slot_member; // [L][K]
     std::vector<uint64_t> span_masks;
     std::vector<uint32_t> span_kranges;
     const FwdVariant *variant = nullptr;
@@ -845,7 +870,9 @@ struct spdy_plan {
     unsigned char *d_blob = nullptr;
     int32_t *d_times = nullptr;
     LayerDesc *d_layers = nullptr;
-    TapRange *d_taps = nullptr;
+    TapRange *d_slots = nullptr;
+    uint8_t *d_slot_ptr = nullptr;
+    uint8_t *d_slot_member = nullptr;
     unsigned long long *d_masks = nullptr;
     unsigned *d_kranges = nullptr;
     int32_t *d_status = nullptr;
@@ -922,6 +949,51 @@ int build_bands(spdy_plan *p)
     return SPDY_OK;
 }
 
+// Shift slots of every layer (see TapRange).  With `merge` the usable choices of a layer are
+// grouped by time, slots in ascending time order; without it slot u is choice u.
+void build_slots(spdy_plan *p, bool merge)
+{
+    const int L = p->L, K = p->K;
+    p->slots.assign(static_cast<size_t>(L) * K, TapRange{0, -1});
+    p->slot_ptr.assign(static_cast<size_t>(L) * (K + 1), 0);
+    p->slot_member.assign(static_cast<size_t>(L) * K, 0);
+    p->distinct_updates = 0;
+    std::vector<int> order(K);
+    for (int l = 0; l < L; ++l) {
+        const TapRange *taps = &p->taps[static_cast<size_t>(l) * K];
+        TapRange *slots = &p->slots[static_cast<size_t>(l) * K];
+        uint8_t *ptr = &p->slot_ptr[static_cast<size_t>(l) * (K + 1)];
+        uint8_t *member = &p->slot_member[static_cast<size_t>(l) * K];
+        int nslots = 0, nmembers = 0;
+        if (!merge) {
+            for (int k = 0; k < K; ++k) {
+                slots[k] = taps[k];
+                ptr[k] = static_cast<uint8_t>(k);
+                member[k] = static_cast<uint8_t>(k);
+            }
+            nslots = nmembers = K;
+        } else {
+            int usable = 0;
+            for (int k = 0; k < K; ++k)
+                if (taps[k].b >= taps[k].a) order[usable++] = k;
+            std::stable_sort(order.begin(), order.begin() + usable,
+                             [&](int x, int y) { return taps[x].a < taps[y].a; });
+            for (int i = 0; i < usable; ++i) {
+                const int k = order[i];
+                if (nslots == 0 || slots[nslots - 1].a != taps[k].a) {
+                    ptr[nslots] = static_cast<uint8_t>(nmembers);
+                    slots[nslots++] = taps[k];  // equal times have equal ranges
+                }
+                member[nmembers++] = static_cast<uint8_t>(k);
+            }
+        }
+        for (int u = nslots; u <= K; ++u) ptr[u] = static_cast<uint8_t>(nmembers);
+        p->layers[l].nslots = nslots;
+        for (int u = 0; u < nslots; ++u)
+            if (slots[u].b >= slots[u].a) p->distinct_updates += slots[u].b - slots[u].a + 1;
+    }
+}
+
 // Per-layer pass shape for a CTA of `threads` threads, row offsets, table pitch and issued work.
 // A layer of `width` cells is covered in `rounds` rounds of NWARPS warp passes; the cells per lane
 // (cpl <= RMAX) are chosen so that the passes of a round are as full as possible, which keeps the
@@ -955,8 +1027,8 @@ int layout_table(spdy_plan *p, int threads, double *efficiency)
         for (int64_t sp = 0; sp < nspans; ++sp) {
             const int64_t s = sp * span;
             uint64_t words[4] = {0, 0, 0, 0};
-            for (int k = 0; k < p->K; ++k) {
-                const TapRange tr = p->taps[static_cast<size_t>(l) * p->K + k];
+            for (int k = 0; k < ld.nslots; ++k) {
+                const TapRange tr = p->slots[static_cast<size_t>(l) * p->K + k];
                 if (tr.b >= tr.a && s + span > tr.a && s <= tr.b) {
                     words[k >> 6] |= 1ULL << (k & 63);
                     p->issued_updates += span;
@@ -964,7 +1036,7 @@ int layout_table(spdy_plan *p, int threads, double *efficiency)
             }
             for (int w = 0; w < mw; ++w) p->span_masks.push_back(words[w]);
             int k_lo = 0, k_hi = 0, count = 0;
-            for (int k = 0; k < p->K; ++k) {
+            for (int k = 0; k < ld.nslots; ++k) {
                 if (words[k >> 6] >> (k & 63) & 1) {
                     if (count == 0) k_lo = k;
                     k_hi = k + 1;
@@ -1005,8 +1077,8 @@ int layout_cluster(spdy_plan *p, int threads, int C)
         const int64_t slice = round_up((width + C - 1) / C, 32);
         max_slice = std::max(max_slice, slice);
         int64_t amax = 0;
-        for (int k = 0; k < p->K; ++k) {
-            const TapRange tr = p->taps[static_cast<size_t>(l) * p->K + k];
+        for (int k = 0; k < ld.nslots; ++k) {
+            const TapRange tr = p->slots[static_cast<size_t>(l) * p->K + k];
             if (tr.b >= tr.a) amax = std::max<int64_t>(amax, tr.a);
         }
         for (int r = 0; r < C; ++r) {
@@ -1036,8 +1108,8 @@ int layout_cluster(spdy_plan *p, int threads, int C)
                 const int64_t s0 = lo + sp * span;
                 uint64_t words[4] = {0, 0, 0, 0};
                 int k_lo = 0, k_hi = 0, count = 0;
-                for (int k = 0; k < p->K; ++k) {
-                    const TapRange tr = p->taps[static_cast<size_t>(l) * p->K + k];
+                for (int k = 0; k < ld.nslots; ++k) {
+                    const TapRange tr = p->slots[static_cast<size_t>(l) * p->K + k];
                     if (tr.b >= tr.a && s0 + span > tr.a && s0 <= tr.b) {
                         words[k >> 6] |= 1ULL << (k & 63);
                         p->issued_updates += span;
@@ -1129,6 +1201,7 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
         if (!(row_mode || arg_mode)) return SPDY_ERR_INVALID_ARG;
         if (row_mode != (p->table_format == SPDY_TABLE_ROW_F32)) return SPDY_ERR_INVALID_ARG;
     }
+    build_slots(p, p->mode == MODE_ROW || p->mode == MODE_ROW2);
     p->cluster = 1;
     if (opts && opts->cluster != 0 && opts->cluster != 1 && opts->cluster != 2 && opts->cluster != 4 &&
         opts->cluster != 8)
@@ -1181,40 +1254,78 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
     return SPDY_OK;
 }
 
+// Where each device table sits inside one 256-byte aligned block of `total` bytes.
+struct TableLayout {
+    size_t times = 0, layers = 0, slots = 0, slot_ptr = 0, slot_member = 0, masks = 0, kranges = 0,
+           status = 0, slices = 0, total = 0;
+};
+
+TableLayout table_layout(const spdy_plan *p)
+{
+    const size_t n = static_cast<size_t>(p->L) * p->K;
+    TableLayout t;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = off;
+        off += static_cast<size_t>(round_up(static_cast<int64_t>(bytes) + 16, 256));
+        return at;
+    };
+    t.times = take(n * sizeof(int32_t));
+    t.layers = take(p->L * sizeof(LayerDesc));
+    t.slots = take(n * sizeof(TapRange));
+    t.slot_ptr = take(static_cast<size_t>(p->L) * (p->K + 1));
+    t.slot_member = take(n);
+    t.masks = take(p->span_masks.size() * sizeof(uint64_t));
+    t.kranges = take(p->span_kranges.size() * sizeof(uint32_t));
+    t.status = take(256);
+    t.slices = take(p->slices.size() * sizeof(SliceDesc));
+    t.total = off;
+    return t;
+}
+
+// Host image of the table block (the status word starts at zero).
+void pack_tables(const spdy_plan *p, const TableLayout &t, std::vector<unsigned char> &host)
+{
+    host.assign(t.total, 0);
+    auto put = [&](size_t at, const void *src, size_t bytes) {
+        if (bytes) std::memcpy(host.data() + at, src, bytes);
+    };
+    put(t.times, p->times.data(), p->times.size() * sizeof(int32_t));
+    put(t.layers, p->layers.data(), p->layers.size() * sizeof(LayerDesc));
+    put(t.slots, p->slots.data(), p->slots.size() * sizeof(TapRange));
+    put(t.slot_ptr, p->slot_ptr.data(), p->slot_ptr.size());
+    put(t.slot_member, p->slot_member.data(), p->slot_member.size());
+    put(t.masks, p->span_masks.data(), p->span_masks.size() * sizeof(uint64_t));
+    put(t.kranges, p->span_kranges.data(), p->span_kranges.size() * sizeof(uint32_t));
+    put(t.slices, p->slices.data(), p->slices.size() * sizeof(SliceDesc));
+}
+
+void bind_tables(spdy_plan *p, const TableLayout &t, unsigned char *base)
+{
+    p->d_times = reinterpret_cast<int32_t *>(base + t.times);
+    p->d_layers = reinterpret_cast<LayerDesc *>(base + t.layers);
+    p->d_slots = reinterpret_cast<TapRange *>(base + t.slots);
+    p->d_slot_ptr = base + t.slot_ptr;
+    p->d_slot_member = base + t.slot_member;
+    p->d_masks = reinterpret_cast<unsigned long long *>(base + t.masks);
+    p->d_kranges = reinterpret_cast<unsigned *>(base + t.kranges);
+    p->d_status = reinterpret_cast<int32_t *>(base + t.status);
+    p->d_slices = reinterpret_cast<SliceDesc *>(base + t.slices);
+}
+
 int upload_tables(spdy_plan *p)
 {
-    const size_t n_times = static_cast<size_t>(p->L) * p->K;
-    const size_t off_layers = round_up(n_times * sizeof(int32_t), 256);
-    const size_t off_taps = off_layers + round_up(p->L * sizeof(LayerDesc), 256);
-    const size_t off_masks = off_taps + round_up(n_times * sizeof(TapRange), 256);
-    const size_t off_kranges = off_masks + round_up(p->span_masks.size() * sizeof(uint64_t) + 8, 256);
-    const size_t off_status = off_kranges + round_up(p->span_kranges.size() * sizeof(uint32_t) + 4, 256);
-    const size_t off_slices = off_status + 256;
-    const size_t total = off_slices + round_up(p->slices.size() * sizeof(SliceDesc) + 32, 256);
-    std::vector<unsigned char> host(total, 0);
-    if (!p->slices.empty())
-        std::memcpy(host.data() + off_slices, p->slices.data(), p->slices.size() * sizeof(SliceDesc));
-    std::memcpy(host.data(), p->times.data(), n_times * sizeof(int32_t));
-    std::memcpy(host.data() + off_layers, p->layers.data(), p->L * sizeof(LayerDesc));
-    std::memcpy(host.data() + off_taps, p->taps.data(), n_times * sizeof(TapRange));
-    if (!p->span_masks.empty())
-        std::memcpy(host.data() + off_masks, p->span_masks.data(), p->span_masks.size() * sizeof(uint64_t));
-    if (!p->span_kranges.empty())
-        std::memcpy(host.data() + off_kranges, p->span_kranges.data(), p->span_kranges.size() * sizeof(uint32_t));
-    cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&p->d_blob), total);
+    const TableLayout t = table_layout(p);
+    std::vector<unsigned char> host;
+    pack_tables(p, t, host);
+    cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&p->d_blob), t.total);
     if (err != cudaSuccess) {
         g_last_cuda_error = static_cast<int>(err);
         p->d_blob = nullptr;
         return err == cudaErrorMemoryAllocation ? SPDY_ERR_NO_MEMORY : SPDY_ERR_CUDA;
     }
-    SPDY_CUDA_TRY(cudaMemcpy(p->d_blob, host.data(), total, cudaMemcpyHostToDevice));
-    p->d_times = reinterpret_cast<int32_t *>(p->d_blob);
-    p->d_layers = reinterpret_cast<LayerDesc *>(p->d_blob + off_layers);
-    p->d_taps = reinterpret_cast<TapRange *>(p->d_blob + off_taps);
-    p->d_masks = reinterpret_cast<unsigned long long *>(p->d_blob + off_masks);
-    p->d_kranges = reinterpret_cast<unsigned *>(p->d_blob + off_kranges);
-    p->d_status = reinterpret_cast<int32_t *>(p->d_blob + off_status);
-    p->d_slices = reinterpret_cast<SliceDesc *>(p->d_blob + off_slices);
+    SPDY_CUDA_TRY(cudaMemcpy(p->d_blob, host.data(), t.total, cudaMemcpyHostToDevice));
+    bind_tables(p, t, p->d_blob);
     return SPDY_OK;
 }
 
@@ -1240,7 +1351,7 @@ struct DeviceGuard {
 
 extern "C" {
 
-int spdy_version(void) { return 1001; }
+int spdy_version(void) { return 1002; }
 
 int spdy_last_cuda_error(void) { return g_last_cuda_error; }
 
@@ -1329,6 +1440,7 @@ int spdy_plan_get_info(const spdy_plan *plan, spdy_plan_info *info)
     info->band_cells = plan->band_cells;
     info->useful_updates = plan->useful_updates;
     info->issued_updates = plan->issued_updates;
+    info->distinct_updates = plan->distinct_updates;
     info->nominal_updates = static_cast<int64_t>(plan->L) * plan->K * plan->B;
     return SPDY_OK;
 }
@@ -1394,7 +1506,9 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
         }
         FwdArgs fa;
         fa.errors = errors_dev;
-        fa.taps = plan->d_taps;
+        fa.slots = plan->d_slots;
+        fa.slot_ptr = plan->d_slot_ptr;
+        fa.slot_member = plan->d_slot_member;
         fa.layers = plan->d_layers;
         fa.span_masks = plan->d_masks;
         fa.span_kranges = plan->d_kranges;
@@ -1684,36 +1798,25 @@ int spdy_solve_batch_static(const float *errors_dev, const int32_t *times_host, 
         return rc;
     }
 
-    // Carve the plan tables out of the front of the scratch.
-    const size_t n_times = static_cast<size_t>(L) * K;
-    const size_t off_layers = round_up(n_times * sizeof(int32_t), 256);
-    const size_t off_taps = off_layers + round_up(L * sizeof(LayerDesc), 256);
-    const size_t off_masks = off_taps + round_up(n_times * sizeof(TapRange), 256);
-    const size_t off_kranges = off_masks + round_up(p->span_masks.size() * sizeof(uint64_t) + 8, 256);
-    const size_t off_status = off_kranges + round_up(p->span_kranges.size() * sizeof(uint32_t) + 4, 256);
-    const size_t off_table = off_status + 256;
+    // The plan tables go to the front of the scratch, the walk-back table behind them.
+    const TableLayout tl = table_layout(p);
+    const size_t off_table = tl.total;
     const size_t one = p->feasible ? spdy_workspace_bytes(p, 1) : 0;
     if (off_table + one > kStaticScratchBytes) {
         spdy_plan_destroy(p);
         return SPDY_ERR_STATIC_LIMIT;
     }
-    p->d_times = reinterpret_cast<int32_t *>(base);
-    p->d_layers = reinterpret_cast<LayerDesc *>(base + off_layers);
-    p->d_taps = reinterpret_cast<TapRange *>(base + off_taps);
-    p->d_masks = reinterpret_cast<unsigned long long *>(base + off_masks);
-    p->d_kranges = reinterpret_cast<unsigned *>(base + off_kranges);
-    p->d_status = reinterpret_cast<int32_t *>(base + off_status);
-    cudaError_t err = cudaSuccess;
-    auto copy = [&](void *dst, const void *src, size_t bytes) {
-        if (err == cudaSuccess && bytes > 0) err = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, stream);
-    };
-    copy(p->d_times, p->times.data(), n_times * sizeof(int32_t));
-    copy(p->d_layers, p->layers.data(), L * sizeof(LayerDesc));
-    copy(p->d_taps, p->taps.data(), n_times * sizeof(TapRange));
-    copy(p->d_masks, p->span_masks.data(), p->span_masks.size() * sizeof(uint64_t));
-    copy(p->d_kranges, p->span_kranges.data(), p->span_kranges.size() * sizeof(uint32_t));
-    // The array keeps the previous call's contents; only the self-check word must start at zero.
-    if (err == cudaSuccess) err = cudaMemsetAsync(p->d_status, 0, 256, stream);
+    std::vector<unsigned char> host;
+    try {
+        pack_tables(p, tl, host);
+    } catch (const std::bad_alloc &) {
+        spdy_plan_destroy(p);
+        return SPDY_ERR_NO_MEMORY;
+    }
+    bind_tables(p, tl, base);
+    // The array keeps the previous call's contents; the image below overwrites every table and
+    // carries a zero self-check word, the only thing that must start at zero.
+    cudaError_t err = cudaMemcpyAsync(base, host.data(), tl.total, cudaMemcpyHostToDevice, stream);
     if (err != cudaSuccess) {
         g_last_cuda_error = static_cast<int>(err);
         cudaStreamSynchronize(stream);

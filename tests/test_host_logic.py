@@ -89,7 +89,21 @@ def test_bands_of_the_named_configs(cfg):
     assert np.array_equal(plo, lo) and np.array_equal(pwidth, width)
     assert info["max_width"] == width.max() and info["band_cells"] == width.sum()
     assert info["nominal_updates"] == wl.L * wl.K * wl.B
-    assert 0 < info["useful_updates"] <= min(info["issued_updates"], info["nominal_updates"] + wl.L * wl.K)
+    assert 0 < info["distinct_updates"] <= info["useful_updates"] <= info["nominal_updates"] + wl.L * wl.K
+    assert info["distinct_updates"] <= info["issued_updates"]
+    # the byte table keeps one slot per choice: nothing is merged
+    arg = binding.Plan(wl.times, wl.B, device=-1, table_format=binding.SPDY_TABLE_ARG_U8).info
+    assert arg["distinct_updates"] == arg["useful_updates"] == info["useful_updates"] <= arg["issued_updates"]
+    # merged work recomputed from the timing table: one shift per distinct usable time of a layer
+    lo_prev, w_prev, distinct = 0, 1, 0
+    for l in range(wl.L):
+        usable = np.unique(wl.times[l][wl.times[l] <= wl.B])
+        for tau in usable:
+            a = int(tau - usable.min())
+            b = min(int(width[l]) - 1, w_prev - 1 + a)
+            distinct += max(0, b - a + 1)
+        w_prev = int(width[l])
+    assert distinct == info["distinct_updates"]
     assert info["smem_bytes"] <= 232448
     assert info["table_bytes_per_candidate"] % 256 == 0
 
@@ -144,4 +158,4 @@ def test_wide_rows_choose_a_cluster():
     small = W.make_workload(2, N=1)
     for c in (2, 4, 8):
         info = binding.Plan(small.times, small.B, device=-1, cluster=c).info
-        assert info["cluster"] == c and info["useful_updates"] <= info["issued_updates"]
+        assert info["cluster"] == c and info["distinct_updates"] <= info["issued_updates"]
