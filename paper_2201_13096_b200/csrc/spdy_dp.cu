@@ -37,7 +37,10 @@ thread_local int g_last_cuda_error = 0;
 // Device-side layout
 // ----------------------------------------------------------------------------------------------
 
-constexpr int RMAX = 16;        // most band cells one lane owns in one pass
+#ifndef SPDY_RMAX
+#define SPDY_RMAX 24
+#endif
+constexpr int RMAX = SPDY_RMAX;  // most band cells one lane owns in one pass (<= 24)
 constexpr int PAD = 32 * RMAX;  // +inf guard cells on either side of a shared-memory row
 
 // How the forward kernel forms a cell and what it stores for the walk back.
@@ -240,10 +243,16 @@ __device__ __forceinline__ void process_span(const float *__restrict__ prev, flo
         if (dense) {
             int k = k_lo;
             if (MODE == MODE_ROW2) {
+                // An odd first slot goes alone so that every pair below is one aligned 16-byte read.
+                if ((k & 1) && k < k_hi) {
+                    const int2 ta = taps[k];
+                    update_min1<RR>(best, base - ta.x, __int_as_float(ta.y));
+                    ++k;
+                }
 #pragma unroll 1
                 for (; k + 1 < k_hi; k += 2) {
-                    const int2 ta = taps[k], tb = taps[k + 1];
-                    update_min2<RR>(best, base - ta.x, __int_as_float(ta.y), base - tb.x, __int_as_float(tb.y));
+                    const int4 t = *reinterpret_cast<const int4 *>(taps + k);
+                    update_min2<RR>(best, base - t.x, __int_as_float(t.y), base - t.z, __int_as_float(t.w));
                 }
             }
 #pragma unroll 1
@@ -347,6 +356,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
     const int warp = tid >> 5;
     constexpr int NWARPS = NT / 32;
     const int L = args.L, K = args.K;
+    const int KS = (K + 1) & ~1;  // slots per staging buffer: even, so that slot pairs are 16-byte aligned
     const int64_t n_local = blockIdx.x;
     const int64_t n = args.n_first + n_local;
     const float *err_n = args.errors + n * L * K;
@@ -362,7 +372,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
     for (int l = 0; l < L; ++l) {
         const float *prev = rows + (l & 1) * args.row_stride + PAD;
         float *cur = rows + ((l + 1) & 1) * args.row_stride + PAD;
-        const int2 *taps = tap_buf + (l & 1) * K;
+        const int2 *taps = tap_buf + (l & 1) * KS;
         const LayerDesc ld = args.layers[l];
 
         // Fetch the next layer's slots early; they are parked in shared memory after the pass.
@@ -380,14 +390,16 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         switch (ld.cpl) {
 #define SPDY_CASE(RR)                                                                          \
     case RR:                                                                                   \
-        for (int span = warp; span < ld.nspans; span += NWARPS)                                \
-            process_span<RR, MODE, false>(prev, cur, taps, __ldg(kranges + span),              \
-                                          masks + span * MW, MW, span * (32 * RR), lane,       \
-                                          row_base, 0);                                        \
+        if constexpr (RR <= RMAX)                                                              \
+            for (int span = warp; span < ld.nspans; span += NWARPS)                            \
+                process_span<RR, MODE, false>(prev, cur, taps, __ldg(kranges + span),          \
+                                              masks + span * MW, MW, span * (32 * RR), lane,   \
+                                              row_base, 0);                                    \
         break;
             SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
             SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
-            SPDY_CASE(13) SPDY_CASE(14) SPDY_CASE(15) SPDY_CASE(16)
+            SPDY_CASE(13) SPDY_CASE(14) SPDY_CASE(15) SPDY_CASE(16) SPDY_CASE(17) SPDY_CASE(18)
+            SPDY_CASE(19) SPDY_CASE(20) SPDY_CASE(21) SPDY_CASE(22) SPDY_CASE(23) SPDY_CASE(24)
 #undef SPDY_CASE
             default: break;
         }
@@ -395,7 +407,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         // passes above wrote +inf from `width` up to nspans*span (those cells saw only +inf
         // sources); PAD more cells of +inf cover the rest.
         for (int i = tid; i < PAD; i += NT) cur[ld.nspans * span_cells + i] = INF;
-        if (have_next) tap_buf[((l + 1) & 1) * K + tid] = next_tap;
+        if (have_next) tap_buf[((l + 1) & 1) * KS + tid] = next_tap;
         __syncthreads();
     }
 
@@ -503,6 +515,7 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
     const int lane = tid & 31;
     const int warp = tid >> 5;
     const int L = args.L, K = args.K;
+    const int KS = (K + 1) & ~1;
     const int64_t n_local = blockIdx.x / C;
     const int64_t n = args.n_first + n_local;
     const float *err_n = args.errors + n * L * K;
@@ -519,7 +532,7 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
     for (int l = 0; l < L; ++l) {
         const SliceDesc sd = cargs.slices[l * C + rank];
         const LayerDesc ld = args.layers[l];
-        const int2 *taps = tap_buf + (l & 1) * K;
+        const int2 *taps = tap_buf + (l & 1) * KS;
         float *out_prev = out + (l & 1) * cargs.out_stride;
         float *out_cur = out + ((l + 1) & 1) * cargs.out_stride;
 
@@ -561,18 +574,20 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
         switch (sd.cpl) {
 #define SPDY_CASE(RR)                                                                             \
     case RR:                                                                                      \
-        for (int span = warp; span < sd.nspans; span += NWARPS)                                   \
-            process_span<RR, MODE, true>(prev, cur, taps, __ldg(kranges + span),                  \
-                                         masks + span * MW, MW, sd.slice_lo + span * (32 * RR),   \
-                                         lane, row_base, sd.slice_hi);                            \
+        if constexpr (RR <= RMAX)                                                                 \
+            for (int span = warp; span < sd.nspans; span += NWARPS)                               \
+                process_span<RR, MODE, true>(prev, cur, taps, __ldg(kranges + span),              \
+                                             masks + span * MW, MW, sd.slice_lo + span * (32 * RR), \
+                                             lane, row_base, sd.slice_hi);                        \
         break;
             SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
             SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
-            SPDY_CASE(13) SPDY_CASE(14) SPDY_CASE(15) SPDY_CASE(16)
+            SPDY_CASE(13) SPDY_CASE(14) SPDY_CASE(15) SPDY_CASE(16) SPDY_CASE(17) SPDY_CASE(18)
+            SPDY_CASE(19) SPDY_CASE(20) SPDY_CASE(21) SPDY_CASE(22) SPDY_CASE(23) SPDY_CASE(24)
 #undef SPDY_CASE
             default: break;
         }
-        if (have_next) tap_buf[((l + 1) & 1) * K + tid] = next_tap;
+        if (have_next) tap_buf[((l + 1) & 1) * KS + tid] = next_tap;
         prev_width = ld.width;
         cluster.sync();  // slices of row l+1 complete everywhere; row l no longer needed
     }
@@ -1049,7 +1064,7 @@ int layout_table(spdy_plan *p, int threads, double *efficiency)
     }
     p->pitch = off;
     p->row_stride = static_cast<int32_t>(round_up(max_extent, 32) + 2 * PAD);
-    p->smem_bytes = 2LL * p->row_stride * 4 + 2LL * p->K * 8;
+    p->smem_bytes = 2LL * p->row_stride * 4 + 2LL * ((p->K + 1) & ~1) * 8;
     if (efficiency) *efficiency = lanes_cells > 0 ? static_cast<double>(p->band_cells) / lanes_cells : 0.0;
     return SPDY_OK;
 }
@@ -1129,7 +1144,7 @@ int layout_cluster(spdy_plan *p, int threads, int C)
     p->out_stride = static_cast<int32_t>(round_up(max_slice, 32));
     p->win_stride = static_cast<int32_t>(round_up(max_win, 32));
     p->row_stride = 0;
-    p->smem_bytes = (2LL * p->out_stride + p->win_stride) * 4 + 2LL * p->K * 8;
+    p->smem_bytes = (2LL * p->out_stride + p->win_stride) * 4 + 2LL * ((p->K + 1) & ~1) * 8;
     return SPDY_OK;
 }
 
