@@ -41,7 +41,6 @@ thread_local int g_last_cuda_error = 0;
 #define SPDY_RMAX 24
 #endif
 constexpr int RMAX = SPDY_RMAX;  // most band cells one lane owns in one pass (<= 24)
-constexpr int PAD = 32 * RMAX;  // +inf guard cells on either side of a shared-memory row
 
 // How the forward kernel forms a cell and what it stores for the walk back.
 enum ForwardMode {
@@ -95,6 +94,7 @@ struct FwdArgs {
     int64_t n_first;          // first candidate of this wave
     int32_t L, K;
     int32_t row_stride;       // floats per shared-memory row buffer
+    int32_t pad;              // +inf guard cells on either side of a row: 32 * the largest cells-per-lane
 };
 
 __device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
@@ -210,7 +210,7 @@ __device__ __forceinline__ void update_arg_pred(float (&best)[RR], float (&idxf)
 
 // One warp pass: the 32*RR band cells starting at s (lane i owns cells s + i, s + i + 32, ...),
 // so every shared-memory access is lane-consecutive (conflict-free) whatever the shift.  Both row
-// buffers carry PAD cells of +inf on either side of the band: a pass that only partly overlaps a
+// buffers carry `pad` cells of +inf (the widest pass of the plan) on either side of the band: a pass that only partly overlaps a
 // choice's range reads +inf for the cells outside it and needs no per-cell bounds check.  Which
 // choices overlap the pass at all is known on the host.  `krange` = k_lo | k_hi << 8 | dense << 16:
 // the overlapping choices lie in [k_lo, k_hi); when they are all of that range (dense, the usual
@@ -343,7 +343,10 @@ __device__ __forceinline__ void process_span(const float *__restrict__ prev, flo
     }
 }
 
-template <int MODE, int NT, int MINB>
+// RCAP: the largest cells-per-lane this instantiation can run.  The registers a kernel needs grow
+// with the largest unrolled pass, so plans whose rows are narrow (few cells per lane) use the
+// RCAP = 8 build, which fits twice as many CTAs per SM.
+template <int MODE, int NT, int MINB, int RCAP>
 __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs args)
 {
     constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
@@ -366,6 +369,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
     for (int i = tid; i < 2 * args.row_stride; i += NT) rows[i] = INF;
     for (int u = tid; u < args.layers[0].nslots; u += NT) tap_buf[u] = stage_slot(args, err_n, 0, u);
     __syncthreads();
+    const int PAD = args.pad;
     if (tid == 0) rows[PAD] = 0.0f;
     __syncthreads();
 
@@ -390,7 +394,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         switch (ld.cpl) {
 #define SPDY_CASE(RR)                                                                          \
     case RR:                                                                                   \
-        if constexpr (RR <= RMAX)                                                              \
+        if constexpr (RR <= RMAX && RR <= RCAP)                                                \
             for (int span = warp; span < ld.nspans; span += NWARPS)                            \
                 process_span<RR, MODE, false>(prev, cur, taps, __ldg(kranges + span),          \
                                               masks + span * MW, MW, span * (32 * RR), lane,   \
@@ -795,22 +799,19 @@ using FwdKernel = void (*)(const FwdArgs);
 struct FwdVariant {
     int mode;
     int threads;
-    int min_blocks;
+    int rcap;
     FwdKernel fn;
 };
 
-#define SPDY_VARIANT(MODE, NT, MINB) \
-    FwdVariant { MODE, NT, MINB, spdy_forward_kernel<MODE, NT, MINB> }
+#define SPDY_VARIANT(MODE, NT, MINB, RCAP) \
+    FwdVariant { MODE, NT, RCAP, spdy_forward_kernel<MODE, NT, MINB, RCAP> }
+#define SPDY_VARIANTS(MODE)                                                                        \
+    SPDY_VARIANT(MODE, 128, 4, RMAX), SPDY_VARIANT(MODE, 256, 2, RMAX), SPDY_VARIANT(MODE, 512, 1, RMAX), \
+    SPDY_VARIANT(MODE, 1024, 1, 16), SPDY_VARIANT(MODE, 128, 6, 8), SPDY_VARIANT(MODE, 256, 3, 8),       \
+    SPDY_VARIANT(MODE, 512, 1, 8), SPDY_VARIANT(MODE, 1024, 1, 8)
 
 const FwdVariant kVariants[] = {
-    SPDY_VARIANT(MODE_ARG, 128, 4),      SPDY_VARIANT(MODE_ARG, 256, 3),
-    SPDY_VARIANT(MODE_ARG, 512, 1),      SPDY_VARIANT(MODE_ARG, 1024, 1),
-    SPDY_VARIANT(MODE_ARG_PRED, 128, 4), SPDY_VARIANT(MODE_ARG_PRED, 256, 3),
-    SPDY_VARIANT(MODE_ARG_PRED, 512, 1), SPDY_VARIANT(MODE_ARG_PRED, 1024, 1),
-    SPDY_VARIANT(MODE_ROW, 128, 4),      SPDY_VARIANT(MODE_ROW, 256, 3),
-    SPDY_VARIANT(MODE_ROW, 512, 1),      SPDY_VARIANT(MODE_ROW, 1024, 1),
-    SPDY_VARIANT(MODE_ROW2, 128, 4),     SPDY_VARIANT(MODE_ROW2, 256, 3),
-    SPDY_VARIANT(MODE_ROW2, 512, 1),     SPDY_VARIANT(MODE_ROW2, 1024, 1),
+    SPDY_VARIANTS(MODE_ARG), SPDY_VARIANTS(MODE_ARG_PRED), SPDY_VARIANTS(MODE_ROW), SPDY_VARIANTS(MODE_ROW2),
 };
 
 using ClusterKernel = void (*)(const ClusterArgs);
@@ -837,10 +838,14 @@ const ClusterVariant *find_cluster_variant(int mode, int threads)
     return nullptr;
 }
 
-const FwdVariant *find_variant(int mode, int threads)
+// A CTA of 1024 threads leaves 64 registers per thread: not enough for 24 cells per lane.
+inline int cells_per_lane_cap(int threads) { return threads >= 1024 ? (RMAX < 16 ? RMAX : 16) : RMAX; }
+
+const FwdVariant *find_variant(int mode, int threads, int max_cpl)
 {
+    const int rcap = max_cpl <= 8 ? 8 : cells_per_lane_cap(threads);
     for (const FwdVariant &v : kVariants)
-        if (v.mode == mode && v.threads == threads) return &v;
+        if (v.mode == mode && v.threads == threads && v.rcap == rcap) return &v;
     return nullptr;
 }
 
@@ -863,7 +868,7 @@ struct spdy_plan {
     int ctas_per_sm = 0;
     int sm_count = 148;
     int64_t smem_bytes = 0;
-    int32_t row_stride = 0;
+    int32_t row_stride = 0, pad = 0;
     int64_t pitch = 0;  // table cells per candidate
     int64_t band_cells = 0, useful_updates = 0, distinct_updates = 0, issued_updates = 0;
     int32_t max_width = 0;
@@ -1020,21 +1025,23 @@ int layout_table(spdy_plan *p, int threads, double *efficiency)
     p->span_masks.clear();
     p->span_kranges.clear();
     int64_t off = 0, lanes_cells = 0;
-    int64_t max_extent = 0;
+    int64_t max_extent = 0, max_cpl = 1;
     p->issued_updates = 0;
     for (int l = 0; l < p->L; ++l) {
         LayerDesc &ld = p->layers[l];
         if (off > 0xffffffffLL) return SPDY_ERR_UNSUPPORTED;
         ld.rowoff = static_cast<uint32_t>(off);
         const int64_t width = ld.width;
-        const int64_t per_round = 32LL * nwarps * RMAX;
+        const int64_t rmax = cells_per_lane_cap(threads);
+        const int64_t per_round = 32LL * nwarps * rmax;
         const int64_t rounds = std::max<int64_t>(1, (width + per_round - 1) / per_round);
         int64_t cpl = (width + 32LL * nwarps * rounds - 1) / (32LL * nwarps * rounds);
-        cpl = std::min<int64_t>(RMAX, std::max<int64_t>(1, cpl));
+        cpl = std::min<int64_t>(rmax, std::max<int64_t>(1, cpl));
         const int64_t span = 32 * cpl;
         const int64_t nspans = (width + span - 1) / span;
         ld.cpl = static_cast<int32_t>(cpl);
         ld.nspans = static_cast<int32_t>(nspans);
+        max_cpl = std::max(max_cpl, cpl);
         max_extent = std::max(max_extent, nspans * span);
         off += round_up(nspans * span, 128);
         lanes_cells += ((nspans + nwarps - 1) / nwarps) * nwarps * span;
@@ -1063,7 +1070,8 @@ int layout_table(spdy_plan *p, int threads, double *efficiency)
         }
     }
     p->pitch = off;
-    p->row_stride = static_cast<int32_t>(round_up(max_extent, 32) + 2 * PAD);
+    p->pad = static_cast<int32_t>(32 * max_cpl);
+    p->row_stride = static_cast<int32_t>(round_up(max_extent, 32) + 2 * p->pad);
     p->smem_bytes = 2LL * p->row_stride * 4 + 2LL * ((p->K + 1) & ~1) * 8;
     if (efficiency) *efficiency = lanes_cells > 0 ? static_cast<double>(p->band_cells) / lanes_cells : 0.0;
     return SPDY_OK;
@@ -1253,7 +1261,7 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
     int rc = layout_table(p, best_threads, nullptr);
     if (rc != SPDY_OK) return rc;
     p->threads = best_threads;
-    p->variant = find_variant(p->mode, best_threads);
+    p->variant = find_variant(p->mode, best_threads, p->pad / 32);
     if (!p->variant) return SPDY_ERR_INVALID_ARG;
     const int64_t by_smem = std::max<int64_t>(1, smem_per_sm / (p->smem_bytes + 1024));
     p->ctas_per_sm = static_cast<int>(std::min<int64_t>(by_smem, 2048 / best_threads));
@@ -1535,6 +1543,7 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
         fa.L = plan->L;
         fa.K = plan->K;
         fa.row_stride = plan->row_stride;
+        fa.pad = plan->pad;
         // Grid x is limited to 2^31-1 CTAs, far above any wave that fits in memory.
         if (plan->cluster > 1) {
             ClusterArgs ca;
