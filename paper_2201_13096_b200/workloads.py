@@ -31,6 +31,10 @@ __all__ = [
     "make_workload",
     "paper_shaped_errors",
     "tiny_random_instance",
+    "sensitivity_samples",
+    "mutation_draws",
+    "synthetic_calibration_loss",
+    "float_times",
     "CONFIG_NAMES",
 ]
 
@@ -247,3 +251,61 @@ def iter_sweep_points() -> Iterator[tuple[int, int]]:
         yield n, 10000
     for b in (1000, 100000):
         yield 4096, b
+
+
+# ---------------------------------------------------------------------------------------------
+# Inputs of the coefficient search (Section 3.3 / Algorithm 4).  The random numbers the search
+# draws are made here, so that every implementation is fed the same ones; none of the search's
+# own steps live in this module.
+# ---------------------------------------------------------------------------------------------
+
+def sensitivity_samples(seed: int, L: int, count: int) -> np.ndarray:
+    """``count`` coefficient vectors uniform in [0, 1]^L (fp32): the samples of Algorithm 4's first loop."""
+    return np.random.default_rng([seed, 1]).uniform(0.0, 1.0, size=(count, L)).astype(np.float32)
+
+
+def mutation_draws(seed: int, L: int):
+    """``draws(d, j)`` -> (indices [d] without repetition, values [d] uniform in [0, 1], fp32): what
+    trial j of neighbourhood size d of Algorithm 4 resamples.  Every (d, j) has its own
+    counter-seeded generator, so the result does not depend on the order of the calls."""
+
+    def draws(d: int, j: int):
+        rng = np.random.default_rng([seed, 2, int(d), int(j)])
+        idx = rng.choice(L, size=int(d), replace=False).astype(np.int64)
+        val = rng.uniform(0.0, 1.0, size=int(d)).astype(np.float32)
+        return idx, val
+
+    return draws
+
+
+def synthetic_calibration_loss(seed: int, L: int, K: int, s_max: float = 0.99):
+    """Stand-in for the calibration loss of a stitched model (Section 3.4 needs the paper's models and
+    data, which are not available): a fixed, deterministic function of the profile that is not
+    additive over layers - per-layer convex penalties plus a coupling of neighbouring layers.
+    An infeasible profile (bytes 0xFF) scores +inf.  Returns ``loss(profile) -> float``."""
+    rng = np.random.default_rng([seed, 3])
+    w = rng.lognormal(0.0, 1.0, size=L)
+    s = sparsity_levels(K, s_max) if K >= 3 else np.linspace(0.0, s_max, K)
+    g = s * s / (1.0 - 0.9 * s)
+    couple = 0.25 * np.sqrt(w[:-1] * w[1:]) if L > 1 else np.zeros(0)
+
+    def loss(profile) -> float:
+        p = np.asarray(profile).astype(np.int64)
+        if (p >= K).any():
+            return float("inf")
+        val = float(np.dot(w, g[p]))
+        if L > 1:
+            val += float(np.dot(couple, s[p[:-1]] * s[p[1:]]))
+        return val
+
+    return loss
+
+
+def float_times(cfg: int, seed_shift: int = 0):
+    """Real-valued layer timings (seconds, fp64) [L][K] of a named config before discretisation,
+    with the dense total; inputs of the discretisation helpers."""
+    wl = make_workload(cfg, N=1, seed_shift=seed_shift)
+    rng = np.random.default_rng([4000 + cfg, seed_shift])
+    scale = 1e-4 * (1.0 + rng.uniform())  # seconds per bucket, arbitrary
+    t = wl.times.astype(np.float64) * scale * (1.0 + 1e-3 * rng.uniform(-1.0, 1.0, size=wl.times.shape))
+    return t, float(t[:, 0].sum())
