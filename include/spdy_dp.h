@@ -154,6 +154,56 @@ int spdy_solve_batch_host(spdy_plan *plan, const float *errors_host, int64_t N,
                           void *cuda_stream);
 
 /*
+ * The same path with the errors of the search's error model (Section 3.3, Eq. 4) instead of a table:
+ *   errors[n][l][i] = coeffs[n][l] * (i / (K - 1))^2,   i = 0 .. K-1 the choice index,
+ * formed inside the kernels as ONE fp32 round-to-nearest multiply of the coefficient with
+ * fp32((i / (K - 1))^2) (the square taken in fp64 and rounded once; K = 1 gives 0).  This is what one
+ * evaluation of Algorithm 4 submits: a candidate is L coefficients rather than L*K errors, so the
+ * input shrinks K-fold.  Results are bit-identical to spdy_solve_batch on the table that
+ * spdy_quadratic_errors writes for the same coefficients.
+ *   coeffs_dev   device, [N][L] fp32 (the paper draws them from [0, 1]; any finite value is accepted).
+ * Everything else as for spdy_solve_batch / spdy_solve_batch_host.
+ */
+int spdy_solve_batch_coeffs(const spdy_plan *plan, const float *coeffs_dev, int64_t N,
+                            uint8_t *profile_dev, float *cost_dev, int32_t *time_used_dev,
+                            void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
+int spdy_solve_batch_coeffs_host(spdy_plan *plan, const float *coeffs_host, int64_t N,
+                                 uint8_t *profile_host, float *cost_host, int32_t *time_used_host,
+                                 void *cuda_stream);
+
+/*
+ * Eq. 4 written out: errors_dev[n][l][i] = coeffs_dev[n][l] * (i / (K - 1))^2 with the arithmetic stated
+ * above.  Device pointers on the current device ([N][L] in, [N][L][K] out), asynchronous on
+ * `cuda_stream`.  INVALID_ARG on null pointers or sizes < 1 (N = 0 is a no-op).
+ */
+int spdy_quadratic_errors(const float *coeffs_dev, int64_t N, int32_t L, int32_t K, float *errors_dev,
+                          void *cuda_stream);
+
+/*
+ * Host-side helpers around the path (no GPU work).
+ *
+ * spdy_time_target: the execution-time target of a speedup target X (Section 3.1):
+ *   T = T_dense / X - T_base, T_base the run time of everything pruning does not touch.
+ *
+ * spdy_bucketize_times: time discretisation of Section 3.2 - B buckets of width T / B, so that the
+ *   budget T becomes B.  out[l][k] = round(times[l][k] * B / T) in fp64, to the nearest integer with
+ *   halves away from zero (SPDY_ROUND_NEAREST) or upwards (SPDY_ROUND_UP; then a profile within B
+ *   buckets is within T in real time).  times_host [L][K] fp64 >= 0, out_host [L][K] int32, both host.
+ *   INVALID_ARG on null, T <= 0, B < 1, a negative or non-finite time, or a result beyond int32.
+ *
+ * spdy_uniform_profile: the "uniform" baseline of Section 4 - the lowest choice index k (choices in
+ *   order of increasing sparsity) such that every layer at choice k fits the budget B; layers flagged
+ *   in keep_dense_host ([L] bytes, may be NULL) stay at choice 0.  *choice_out = k or -1 if none fits,
+ *   *total_out (may be NULL) = that profile's total time or -1.  times_host [L][K] int32 >= 0.
+ */
+typedef enum spdy_rounding { SPDY_ROUND_NEAREST = 0, SPDY_ROUND_UP = 1 } spdy_rounding;
+double spdy_time_target(double t_dense, double speedup, double t_base);
+int spdy_bucketize_times(const double *times_host, int32_t L, int32_t K, double T, int32_t B, int32_t rounding,
+                         int32_t *out_host);
+int spdy_uniform_profile(const int32_t *times_host, int32_t L, int32_t K, int32_t B, const uint8_t *keep_dense_host,
+                         int32_t *choice_out, int64_t *total_out);
+
+/*
  * One-shot form of the whole path: errors[N][L][K], times[L][K], budget B -> profile, cost,
  * time_used, all device pointers on the current device except nothing else.  Reads times back to
  * the host, builds a transient plan, allocates and frees its own workspace, and waits for the

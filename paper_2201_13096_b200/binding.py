@@ -22,6 +22,8 @@ EXPORTS = (
     "spdy_workspace_bytes", "spdy_solve_batch", "spdy_solve_batch_host", "spdy_solve_batch_simple",
     "spdy_plan_check_status", "spdy_plan_enable_timing", "spdy_plan_last_timing",
     "spdy_solve_batch_static", "spdy_static_scratch_bytes", "spdy_strerror", "spdy_last_cuda_error", "spdy_version",
+    "spdy_solve_batch_coeffs", "spdy_solve_batch_coeffs_host", "spdy_quadratic_errors",
+    "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile",
 )
 
 
@@ -83,6 +85,18 @@ def _load():
     lib.spdy_solve_batch.argtypes = [vp, vp, i64, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.spdy_solve_batch_host.restype = ctypes.c_int
     lib.spdy_solve_batch_host.argtypes = [vp, vp, i64, vp, vp, vp, vp]
+    lib.spdy_solve_batch_coeffs.restype = ctypes.c_int
+    lib.spdy_solve_batch_coeffs.argtypes = [vp, vp, i64, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.spdy_solve_batch_coeffs_host.restype = ctypes.c_int
+    lib.spdy_solve_batch_coeffs_host.argtypes = [vp, vp, i64, vp, vp, vp, vp]
+    lib.spdy_quadratic_errors.restype = ctypes.c_int
+    lib.spdy_quadratic_errors.argtypes = [vp, i64, i32, i32, vp, vp]
+    lib.spdy_time_target.restype = ctypes.c_double
+    lib.spdy_time_target.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double]
+    lib.spdy_bucketize_times.restype = ctypes.c_int
+    lib.spdy_bucketize_times.argtypes = [vp, i32, i32, ctypes.c_double, i32, i32, vp]
+    lib.spdy_uniform_profile.restype = ctypes.c_int
+    lib.spdy_uniform_profile.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i64)]
     lib.spdy_solve_batch_simple.restype = ctypes.c_int
     lib.spdy_solve_batch_simple.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.spdy_plan_check_status.restype = ctypes.c_int
@@ -272,3 +286,94 @@ def solve_batch_static(errors, times, B: int, profile=None, cost=None, time_used
                                            time_used.data_ptr(), _stream_handle(stream)),
            "spdy_solve_batch_static")
     return profile, cost, time_used
+
+
+def solve_batch_coeffs(plan: Plan, coeffs, profile=None, cost=None, time_used=None, workspace=None,
+                       stream=None):
+    """``spdy_solve_batch_coeffs``: like ``solve_batch`` with Eq. 4's sensitivity coefficients
+    (contiguous CUDA fp32 tensor [N][L]) in place of an error table."""
+    import torch
+
+    if not (coeffs.is_cuda and coeffs.dtype == torch.float32 and coeffs.is_contiguous()):
+        raise ValueError("coeffs must be a contiguous CUDA float32 tensor")
+    if coeffs.dim() != 2 or coeffs.shape[1] != plan.L:
+        raise ValueError("coeffs must be [N][L] matching the plan")
+    N = int(coeffs.shape[0])
+    dev = coeffs.device
+    if profile is None:
+        profile = torch.empty((N, plan.L), dtype=torch.uint8, device=dev)
+    if cost is None:
+        cost = torch.empty(N, dtype=torch.float32, device=dev)
+    if time_used is None:
+        time_used = torch.empty(N, dtype=torch.int32, device=dev)
+    if workspace is None:
+        need = plan.workspace_bytes(N)
+        if plan._ws is None or plan._ws.numel() < need or plan._ws.device != dev:
+            plan._ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        workspace = plan._ws
+    _check(_load().spdy_solve_batch_coeffs(plan._h, coeffs.data_ptr(), N, profile.data_ptr(),
+                                           cost.data_ptr(), time_used.data_ptr(), workspace.data_ptr(),
+                                           workspace.numel() * workspace.element_size(),
+                                           _stream_handle(stream)), "spdy_solve_batch_coeffs")
+    return profile, cost, time_used
+
+
+def solve_batch_coeffs_host(plan: Plan, coeffs, profile=None, cost=None, time_used=None, stream=None):
+    """``spdy_solve_batch_coeffs_host``: coefficients [N][L] and outputs in host memory (NumPy or
+    pinned torch CPU tensors), copies included."""
+    def addr(x):
+        return x.ctypes.data if isinstance(x, np.ndarray) else x.data_ptr()
+
+    if isinstance(coeffs, np.ndarray):
+        coeffs = np.ascontiguousarray(coeffs, dtype=np.float32)
+    N = int(coeffs.shape[0])
+    if profile is None:
+        profile = np.empty((N, plan.L), np.uint8)
+    if cost is None:
+        cost = np.empty(N, np.float32)
+    if time_used is None:
+        time_used = np.empty(N, np.int32)
+    _check(_load().spdy_solve_batch_coeffs_host(plan._h, addr(coeffs), N, addr(profile), addr(cost),
+                                                addr(time_used), _stream_handle(stream)),
+           "spdy_solve_batch_coeffs_host")
+    return profile, cost, time_used
+
+
+def quadratic_errors(coeffs, K: int, stream=None):
+    """``spdy_quadratic_errors``: Eq. 4's error table [N][L][K] for coefficients [N][L] (CUDA fp32)."""
+    import torch
+
+    N, L = (int(x) for x in coeffs.shape)
+    out = torch.empty((N, L, int(K)), dtype=torch.float32, device=coeffs.device)
+    _check(_load().spdy_quadratic_errors(coeffs.data_ptr(), N, L, int(K), out.data_ptr(),
+                                         _stream_handle(stream)), "spdy_quadratic_errors")
+    return out
+
+
+def time_target(t_dense: float, speedup: float, t_base: float = 0.0) -> float:
+    """``spdy_time_target``: T_dense / X - T_base."""
+    return float(_load().spdy_time_target(float(t_dense), float(speedup), float(t_base)))
+
+
+def bucketize_times(times, T: float, B: int, rounding: str = "nearest") -> np.ndarray:
+    """``spdy_bucketize_times``: real layer times [L][K] -> int32 buckets of width T / B."""
+    t = np.ascontiguousarray(np.asarray(times), dtype=np.float64)
+    if t.ndim != 2:
+        raise ValueError("times must be [L][K]")
+    mode = {"nearest": 0, "up": 1}[rounding]
+    out = np.empty(t.shape, np.int32)
+    _check(_load().spdy_bucketize_times(t.ctypes.data_as(ctypes.c_void_p), int(t.shape[0]), int(t.shape[1]),
+                                        float(T), int(B), mode, out.ctypes.data_as(ctypes.c_void_p)),
+           "spdy_bucketize_times")
+    return out
+
+
+def uniform_profile(times, B: int, keep_dense=None):
+    """``spdy_uniform_profile``: (lowest common choice index that fits B, its total time) or (-1, -1)."""
+    t = np.ascontiguousarray(np.asarray(times), dtype=np.int32)
+    keep = None if keep_dense is None else np.ascontiguousarray(np.asarray(keep_dense), dtype=np.uint8)
+    k, total = ctypes.c_int32(), ctypes.c_int64()
+    _check(_load().spdy_uniform_profile(t.ctypes.data_as(ctypes.c_void_p), int(t.shape[0]), int(t.shape[1]), int(B),
+                                        None if keep is None else keep.ctypes.data_as(ctypes.c_void_p),
+                                        ctypes.byref(k), ctypes.byref(total)), "spdy_uniform_profile")
+    return int(k.value), int(total.value)

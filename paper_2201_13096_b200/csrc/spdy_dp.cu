@@ -14,6 +14,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstdint>
 #include <cstring>
 #include <mutex>
@@ -80,7 +81,9 @@ struct TapRange {
 };
 
 struct FwdArgs {
-    const float *errors;      // [N][L][K]
+    const float *errors;      // [N][L][K], or null when the errors follow from coefficients
+    const float *coeffs;      // [N][L] sensitivity coefficients (Eq. 4), used when errors is null
+    const float *qtab;        // [K]: fp32((i / (K - 1))^2)
     const TapRange *slots;    // [L][K], the first layers[l].nslots of a layer are valid
     const uint8_t *slot_ptr;     // [L][K+1]: members of slot u are slot_member[slot_ptr[u] .. slot_ptr[u+1])
     const uint8_t *slot_member;  // [L][K]: choice indices grouped by slot
@@ -99,17 +102,26 @@ struct FwdArgs {
 
 __device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
 
+// Error of choice k of layer l of candidate n: read from the table, or Eq. 4's c * (k / (K-1))^2 as
+// one fp32 multiply of the coefficient with the pre-rounded square.
+__device__ __forceinline__ float choice_error(const float *errors, const float *coeffs, const float *qtab,
+                                              const int64_t n, const int l, const int k, const int L, const int K)
+{
+    if (errors) return errors[(n * L + l) * K + k];
+    return __fmul_rn(coeffs[n * L + l], qtab[k]);
+}
+
 // (shift, error bits) of slot u of layer l for one candidate: the smallest error among the
 // slot's choices (a single choice unless equal times were merged).
-__device__ __forceinline__ int2 stage_slot(const FwdArgs &args, const float *err_n, const int l, const int u)
+__device__ __forceinline__ int2 stage_slot(const FwdArgs &args, const int64_t n, const int l, const int u)
 {
-    const int K = args.K;
+    const int K = args.K, L = args.L;
     const uint8_t *ptr = args.slot_ptr + static_cast<size_t>(l) * (K + 1);
     const uint8_t *member = args.slot_member + static_cast<size_t>(l) * K;
-    const float *err_l = err_n + static_cast<size_t>(l) * K;
     const int j0 = ptr[u], j1 = ptr[u + 1];
-    float e = err_l[member[j0]];
-    for (int j = j0 + 1; j < j1; ++j) e = fminf(e, err_l[member[j]]);
+    float e = choice_error(args.errors, args.coeffs, args.qtab, n, l, member[j0], L, K);
+    for (int j = j0 + 1; j < j1; ++j)
+        e = fminf(e, choice_error(args.errors, args.coeffs, args.qtab, n, l, member[j], L, K));
     return make_int2(args.slots[static_cast<size_t>(l) * K + u].a, __float_as_int(e));
 }
 
@@ -362,12 +374,11 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
     const int KS = (K + 1) & ~1;  // slots per staging buffer: even, so that slot pairs are 16-byte aligned
     const int64_t n_local = blockIdx.x;
     const int64_t n = args.n_first + n_local;
-    const float *err_n = args.errors + n * L * K;
     const float INF = pos_inf();
 
     // Both buffers start as +inf everywhere; D_0 is +0 at t = 0 (Eq. 3 via a virtual row 0).
     for (int i = tid; i < 2 * args.row_stride; i += NT) rows[i] = INF;
-    for (int u = tid; u < args.layers[0].nslots; u += NT) tap_buf[u] = stage_slot(args, err_n, 0, u);
+    for (int u = tid; u < args.layers[0].nslots; u += NT) tap_buf[u] = stage_slot(args, n, 0, u);
     __syncthreads();
     const int PAD = args.pad;
     if (tid == 0) rows[PAD] = 0.0f;
@@ -383,7 +394,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         // (NT >= K is guaranteed by the host, so one thread per slot suffices.)
         int2 next_tap = make_int2(0, 0);
         const bool have_next = (l + 1 < L) && (tid < args.layers[l + 1].nslots);
-        if (have_next) next_tap = stage_slot(args, err_n, l + 1, tid);
+        if (have_next) next_tap = stage_slot(args, n, l + 1, tid);
 
         unsigned char *row_base = static_cast<unsigned char *>(args.table) +
                                   (n_local * args.pitch + ld.rowoff) * (ROWFMT ? 4 : 1);
@@ -522,12 +533,11 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
     const int KS = (K + 1) & ~1;
     const int64_t n_local = blockIdx.x / C;
     const int64_t n = args.n_first + n_local;
-    const float *err_n = args.errors + n * L * K;
     const float INF = pos_inf();
 
     // Virtual row 0: +0 at t = 0, held in rank 0's first `out` buffer.
     for (int i = tid; i < 2 * cargs.out_stride; i += NT) out[i] = INF;
-    for (int u = tid; u < args.layers[0].nslots; u += NT) tap_buf[u] = stage_slot(args, err_n, 0, u);
+    for (int u = tid; u < args.layers[0].nslots; u += NT) tap_buf[u] = stage_slot(args, n, 0, u);
     __syncthreads();
     if (rank == 0 && tid == 0) out[0] = 0.0f;
     cluster.sync();
@@ -542,7 +552,7 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
 
         int2 next_tap = make_int2(0, 0);
         const bool have_next = (l + 1 < L) && (tid < args.layers[l + 1].nslots);
-        if (have_next) next_tap = stage_slot(args, err_n, l + 1, tid);
+        if (have_next) next_tap = stage_slot(args, n, l + 1, tid);
 
         // Gather the window [q0, q0 + win_len) of the previous row, peer by peer; cells outside
         // the previous band read as +inf.
@@ -661,7 +671,9 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
 }
 
 struct BackArgs {
-    const float *errors;      // [N][L][K]
+    const float *errors;      // [N][L][K], or null (see FwdArgs)
+    const float *coeffs;      // [N][L]
+    const float *qtab;        // [K]
     const int32_t *times;     // [L][K]
     const LayerDesc *layers;  // [L]
     const void *table;
@@ -724,7 +736,6 @@ __global__ void spdy_backtrack_row_kernel(const BackArgs args)
     }
     const float INF = pos_inf();
     const float *D = static_cast<const float *>(args.table) + n_local * args.pitch;
-    const float *err_n = args.errors + n * L * K;
     float target = args.cost[n];
     bool ok = true;
     for (int l = L - 1; l >= 0; --l) {
@@ -750,7 +761,7 @@ __global__ void spdy_backtrack_row_kernel(const BackArgs args)
                 const int64_t src = static_cast<int64_t>(t_rel) - (static_cast<int64_t>(tau) - ld.mn);
                 if (src >= 0 && src < prev_width) {
                     pv = (l == 0) ? 0.0f : D[prev_off + src];
-                    const float v = __fadd_rn(pv, err_n[l * K + k]);
+                    const float v = __fadd_rn(pv, choice_error(args.errors, args.coeffs, args.qtab, n, l, k, L, K));
                     match = (v == target) && (pv < INF);
                 }
             }
@@ -776,6 +787,22 @@ __global__ void spdy_backtrack_row_kernel(const BackArgs args)
         }
     }
     if ((!ok || t != 0) && lane == 0) atomicExch(args.status, 1);
+}
+
+// Eq. 4 written out as a table: errors[n][l][i] = c[n][l] * (i / (K-1))^2, the same fp32 multiply
+// of the coefficient with the pre-rounded square that the solver's coefficient mode performs in place.
+__global__ void spdy_quadratic_errors_kernel(const float *coeffs, float *errors, int64_t total, int32_t K)
+{
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t j = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; j < total; j += stride) {
+        const int i = static_cast<int>(j % K);
+        float q = 0.0f;
+        if (K > 1) {
+            const double r = static_cast<double>(i) / static_cast<double>(K - 1);
+            q = static_cast<float>(r * r);
+        }
+        errors[j] = __fmul_rn(coeffs[j / K], q);
+    }
 }
 
 __global__ void spdy_fill_infeasible_kernel(uint8_t *profile, float *cost, int32_t *time_used,
@@ -873,6 +900,7 @@ struct spdy_plan {
     int64_t band_cells = 0, useful_updates = 0, distinct_updates = 0, issued_updates = 0;
     int32_t max_width = 0;
     std::vector<int32_t> times;
+    std::vector<float> qtab;          // [K] squares of Eq. 4
     std::vector<LayerDesc> layers;
     std::vector<TapRange> taps;       // [L][K] by choice
     std::vector<TapRange> slots;      // [L][K] by shift slot (first layers[l].nslots valid)
@@ -896,6 +924,7 @@ struct spdy_plan {
     unsigned long long *d_masks = nullptr;
     unsigned *d_kranges = nullptr;
     int32_t *d_status = nullptr;
+    float *d_qtab = nullptr;
     // optional event timing of the last solve (three events per wave)
     bool timing = false;
     std::vector<cudaEvent_t> events;
@@ -906,6 +935,16 @@ struct spdy_plan {
 };
 
 namespace {
+
+// Eq. 4's squares (i / (K - 1))^2, formed in fp64 and rounded once to fp32; K = 1 gives 0.
+void fill_qtab(spdy_plan *p)
+{
+    p->qtab.assign(p->K, 0.0f);
+    for (int i = 0; i < p->K && p->K > 1; ++i) {
+        const double r = static_cast<double>(i) / static_cast<double>(p->K - 1);
+        p->qtab[i] = static_cast<float>(r * r);
+    }
+}
 
 int64_t cell_bytes(const spdy_plan *p) { return p->table_format == SPDY_TABLE_ROW_F32 ? 4 : 1; }
 
@@ -1280,7 +1319,7 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
 // Where each device table sits inside one 256-byte aligned block of `total` bytes.
 struct TableLayout {
     size_t times = 0, layers = 0, slots = 0, slot_ptr = 0, slot_member = 0, masks = 0, kranges = 0,
-           status = 0, slices = 0, total = 0;
+           status = 0, slices = 0, qtab = 0, total = 0;
 };
 
 TableLayout table_layout(const spdy_plan *p)
@@ -1302,6 +1341,7 @@ TableLayout table_layout(const spdy_plan *p)
     t.kranges = take(p->span_kranges.size() * sizeof(uint32_t));
     t.status = take(256);
     t.slices = take(p->slices.size() * sizeof(SliceDesc));
+    t.qtab = take(p->qtab.size() * sizeof(float));
     t.total = off;
     return t;
 }
@@ -1321,6 +1361,7 @@ void pack_tables(const spdy_plan *p, const TableLayout &t, std::vector<unsigned 
     put(t.masks, p->span_masks.data(), p->span_masks.size() * sizeof(uint64_t));
     put(t.kranges, p->span_kranges.data(), p->span_kranges.size() * sizeof(uint32_t));
     put(t.slices, p->slices.data(), p->slices.size() * sizeof(SliceDesc));
+    put(t.qtab, p->qtab.data(), p->qtab.size() * sizeof(float));
 }
 
 void bind_tables(spdy_plan *p, const TableLayout &t, unsigned char *base)
@@ -1334,6 +1375,7 @@ void bind_tables(spdy_plan *p, const TableLayout &t, unsigned char *base)
     p->d_kranges = reinterpret_cast<unsigned *>(base + t.kranges);
     p->d_status = reinterpret_cast<int32_t *>(base + t.status);
     p->d_slices = reinterpret_cast<SliceDesc *>(base + t.slices);
+    p->d_qtab = reinterpret_cast<float *>(base + t.qtab);
 }
 
 int upload_tables(spdy_plan *p)
@@ -1374,7 +1416,7 @@ struct DeviceGuard {
 
 extern "C" {
 
-int spdy_version(void) { return 1002; }
+int spdy_version(void) { return 1003; }
 
 int spdy_last_cuda_error(void) { return g_last_cuda_error; }
 
@@ -1414,6 +1456,7 @@ int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int3
     int rc = SPDY_OK;
     try {
         p->times.assign(times_host, times_host + static_cast<size_t>(L) * K);
+        fill_qtab(p);
         rc = build_bands(p);
         DeviceGuard guard;
         if (rc == SPDY_OK && device >= 0) rc = guard.enter(device);
@@ -1485,14 +1528,20 @@ size_t spdy_workspace_bytes(const spdy_plan *plan, int64_t N)
     return static_cast<size_t>(per) * static_cast<size_t>(N);
 }
 
-int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
-                     uint8_t *profile_dev, float *cost_dev, int32_t *time_used_dev,
-                     void *workspace_dev, size_t workspace_bytes, void *cuda_stream)
+}  // extern "C"
+
+namespace {
+
+// The whole path for one batch; exactly one of errors_dev / coeffs_dev is non-null.
+int solve_impl(const spdy_plan *plan, const float *errors_dev, const float *coeffs_dev, int64_t N,
+               uint8_t *profile_dev, float *cost_dev, int32_t *time_used_dev, void *workspace_dev,
+               size_t workspace_bytes, void *cuda_stream)
 {
     if (!plan || plan->device < 0 || N < 0) return SPDY_ERR_INVALID_ARG;
     if (N == 0) return SPDY_OK;
-    if (!errors_dev || !profile_dev || !cost_dev || !time_used_dev) return SPDY_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(errors_dev) % 4 != 0) return SPDY_ERR_INVALID_ARG;
+    const float *input = errors_dev ? errors_dev : coeffs_dev;
+    if (!input || !profile_dev || !cost_dev || !time_used_dev) return SPDY_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(input) % 4 != 0) return SPDY_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     DeviceGuard guard;
     int rc = guard.enter(plan->device);
@@ -1529,6 +1578,8 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
         }
         FwdArgs fa;
         fa.errors = errors_dev;
+        fa.coeffs = coeffs_dev;
+        fa.qtab = plan->d_qtab;
         fa.slots = plan->d_slots;
         fa.slot_ptr = plan->d_slot_ptr;
         fa.slot_member = plan->d_slot_member;
@@ -1573,6 +1624,8 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
 
         BackArgs ba;
         ba.errors = errors_dev;
+        ba.coeffs = coeffs_dev;
+        ba.qtab = plan->d_qtab;
         ba.times = plan->d_times;
         ba.layers = plan->d_layers;
         ba.table = workspace_dev;
@@ -1596,6 +1649,28 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
         if (ev) SPDY_CUDA_TRY(cudaEventRecord(ev[2], stream));
     }
     return SPDY_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
+                     uint8_t *profile_dev, float *cost_dev, int32_t *time_used_dev,
+                     void *workspace_dev, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!errors_dev && N > 0) return SPDY_ERR_INVALID_ARG;
+    return solve_impl(plan, errors_dev, nullptr, N, profile_dev, cost_dev, time_used_dev, workspace_dev,
+                      workspace_bytes, cuda_stream);
+}
+
+int spdy_solve_batch_coeffs(const spdy_plan *plan, const float *coeffs_dev, int64_t N,
+                            uint8_t *profile_dev, float *cost_dev, int32_t *time_used_dev,
+                            void *workspace_dev, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!coeffs_dev && N > 0) return SPDY_ERR_INVALID_ARG;
+    return solve_impl(plan, nullptr, coeffs_dev, N, profile_dev, cost_dev, time_used_dev, workspace_dev,
+                      workspace_bytes, cuda_stream);
 }
 
 int spdy_plan_enable_timing(spdy_plan *plan, int on)
@@ -1644,9 +1719,14 @@ int spdy_plan_check_status(spdy_plan *plan, void *cuda_stream)
     return SPDY_OK;
 }
 
-int spdy_solve_batch_host(spdy_plan *plan, const float *errors_host, int64_t N,
-                          uint8_t *profile_host, float *cost_host, int32_t *time_used_host,
-                          void *cuda_stream)
+}  // extern "C"
+
+namespace {
+
+// Host-buffer form of the path: the input is an error table ([N][L][K]) or, with `coeffs`, Eq. 4's
+// coefficients ([N][L]).
+int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int64_t N,
+                    uint8_t *profile_host, float *cost_host, int32_t *time_used_host, void *cuda_stream)
 {
     if (!plan || plan->device < 0 || N < 0) return SPDY_ERR_INVALID_ARG;
     if (N == 0) return SPDY_OK;
@@ -1656,7 +1736,7 @@ int spdy_solve_batch_host(spdy_plan *plan, const float *errors_host, int64_t N,
     int rc = guard.enter(plan->device);
     if (rc != SPDY_OK) return rc;
 
-    const size_t err_bytes = static_cast<size_t>(N) * plan->L * plan->K * sizeof(float);
+    const size_t err_bytes = static_cast<size_t>(N) * plan->L * (coeffs ? 1 : plan->K) * sizeof(float);
     const size_t off_profile = round_up(err_bytes, 256);
     const size_t off_cost = off_profile + round_up(static_cast<size_t>(N) * plan->L, 256);
     const size_t off_time = off_cost + round_up(static_cast<size_t>(N) * 4, 256);
@@ -1688,12 +1768,92 @@ int spdy_solve_batch_host(spdy_plan *plan, const float *errors_host, int64_t N,
     float *d_cost = reinterpret_cast<float *>(base + off_cost);
     int32_t *d_time = reinterpret_cast<int32_t *>(base + off_time);
     SPDY_CUDA_TRY(cudaMemcpyAsync(d_err, errors_host, err_bytes, cudaMemcpyHostToDevice, stream));
-    rc = spdy_solve_batch(plan, d_err, N, d_profile, d_cost, d_time, base + off_ws, ws_bytes, stream);
+    rc = solve_impl(plan, coeffs ? nullptr : d_err, coeffs ? d_err : nullptr, N, d_profile, d_cost, d_time,
+                    base + off_ws, ws_bytes, stream);
     if (rc != SPDY_OK) return rc;
     SPDY_CUDA_TRY(cudaMemcpyAsync(profile_host, d_profile, static_cast<size_t>(N) * plan->L, cudaMemcpyDeviceToHost, stream));
     SPDY_CUDA_TRY(cudaMemcpyAsync(cost_host, d_cost, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
     SPDY_CUDA_TRY(cudaMemcpyAsync(time_used_host, d_time, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
     SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
+    return SPDY_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int spdy_solve_batch_host(spdy_plan *plan, const float *errors_host, int64_t N,
+                          uint8_t *profile_host, float *cost_host, int32_t *time_used_host,
+                          void *cuda_stream)
+{
+    return solve_host_impl(plan, errors_host, false, N, profile_host, cost_host, time_used_host, cuda_stream);
+}
+
+int spdy_solve_batch_coeffs_host(spdy_plan *plan, const float *coeffs_host, int64_t N,
+                                 uint8_t *profile_host, float *cost_host, int32_t *time_used_host,
+                                 void *cuda_stream)
+{
+    return solve_host_impl(plan, coeffs_host, true, N, profile_host, cost_host, time_used_host, cuda_stream);
+}
+
+int spdy_quadratic_errors(const float *coeffs_dev, int64_t N, int32_t L, int32_t K, float *errors_dev,
+                          void *cuda_stream)
+{
+    if (N < 0 || L < 1 || K < 1) return SPDY_ERR_INVALID_ARG;
+    if (N == 0) return SPDY_OK;
+    if (!coeffs_dev || !errors_dev) return SPDY_ERR_INVALID_ARG;
+    const int64_t total = N * L * K;
+    const int blocks = static_cast<int>(std::min<int64_t>((total + 255) / 256, 148 * 16));
+    spdy_quadratic_errors_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(coeffs_dev, errors_dev, total, K);
+    SPDY_CUDA_TRY(cudaGetLastError());
+    return SPDY_OK;
+}
+
+double spdy_time_target(double t_dense, double speedup, double t_base)
+{
+    return t_dense / speedup - t_base;
+}
+
+int spdy_bucketize_times(const double *times_host, int32_t L, int32_t K, double T, int32_t B, int32_t rounding,
+                         int32_t *out_host)
+{
+    if (!times_host || !out_host || L < 1 || K < 1 || B < 1 || !(T > 0.0) || !std::isfinite(T)) return SPDY_ERR_INVALID_ARG;
+    if (rounding != SPDY_ROUND_NEAREST && rounding != SPDY_ROUND_UP) return SPDY_ERR_INVALID_ARG;
+    const size_t n = static_cast<size_t>(L) * K;
+    for (size_t i = 0; i < n; ++i) {
+        const double t = times_host[i];
+        if (!(t >= 0.0) || !std::isfinite(t)) return SPDY_ERR_INVALID_ARG;
+        const double v = t * static_cast<double>(B) / T;
+        const double r = rounding == SPDY_ROUND_UP ? std::ceil(v) : std::floor(v + 0.5);
+        if (r > 2147483647.0) return SPDY_ERR_INVALID_ARG;
+    }
+    for (size_t i = 0; i < n; ++i) {
+        const double v = times_host[i] * static_cast<double>(B) / T;
+        out_host[i] = static_cast<int32_t>(rounding == SPDY_ROUND_UP ? std::ceil(v) : std::floor(v + 0.5));
+    }
+    return SPDY_OK;
+}
+
+int spdy_uniform_profile(const int32_t *times_host, int32_t L, int32_t K, int32_t B, const uint8_t *keep_dense_host,
+                         int32_t *choice_out, int64_t *total_out)
+{
+    if (!times_host || !choice_out || L < 1 || K < 1 || B < 0) return SPDY_ERR_INVALID_ARG;
+    *choice_out = -1;
+    if (total_out) *total_out = -1;
+    for (size_t i = 0; i < static_cast<size_t>(L) * K; ++i)
+        if (times_host[i] < 0) return SPDY_ERR_INVALID_ARG;
+    for (int k = 0; k < K; ++k) {
+        int64_t total = 0;
+        for (int l = 0; l < L; ++l) {
+            const int use = (keep_dense_host && keep_dense_host[l]) ? 0 : k;
+            total += times_host[static_cast<size_t>(l) * K + use];
+        }
+        if (total <= B) {
+            *choice_out = k;
+            if (total_out) *total_out = total;
+            break;
+        }
+    }
     return SPDY_OK;
 }
 
@@ -1811,6 +1971,7 @@ int spdy_solve_batch_static(const float *errors_dev, const int32_t *times_host, 
     opts.cluster = 1;  // the cluster variant's wider rows would not leave room for a table anyway
     try {
         p->times.assign(times_host, times_host + static_cast<size_t>(L) * K);
+        fill_qtab(p);
         rc = build_bands(p);
         if (rc == SPDY_OK) rc = choose_launch_shape(p, &opts);
     } catch (const std::bad_alloc &) {

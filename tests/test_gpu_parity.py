@@ -234,3 +234,77 @@ def test_cluster_with_ties_and_wide_rows():
     for cluster in (2, 4, 8):
         for fmt in FORMATS:
             assert_same(gpu_solve(wl, fmt, cluster=cluster), ref)
+
+
+def coeff_cases():
+    rng = np.random.default_rng(5)
+    for cfg, N in ((1, 48), (2, 48), (3, 4)):
+        wl = W.make_workload(cfg, N=1)
+        yield wl.times, wl.B, rng.uniform(0.0, 1.0, size=(N, wl.L)).astype(np.float32)
+    wl = W.make_workload(4, N=1, B=1000)
+    yield wl.times, wl.B, rng.uniform(0.0, 1.0, size=(40, wl.L)).astype(np.float32)
+    wl = W.make_workload(2, N=1)
+    c = rng.normal(size=(16, wl.L)).astype(np.float32)  # signed coefficients are accepted too
+    c[0], c[1] = 0.0, 1.0
+    yield wl.times, wl.B, c
+
+
+def test_eq4_error_table_element_by_element():
+    import torch
+
+    rng = np.random.default_rng(6)
+    for K in (1, 2, 3, 5, 42, 64, 255):
+        c = rng.uniform(0.0, 1.0, size=(37, 11)).astype(np.float32)
+        c[0, :4] = [0.0, 1.0, 1e-30, -0.75]
+        got = binding.quadratic_errors(torch.from_numpy(c).cuda(), K).cpu().numpy()
+        assert got.tobytes() == oracle.quadratic_errors(c, K).tobytes()
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_coefficient_input_matches_the_oracle_on_eq4_errors(fmt):
+    """spdy_solve_batch_coeffs forms Eq. 4's errors inside the kernels; the oracle forms the table
+    first and runs the same dynamic program."""
+    import torch
+
+    for times, B, c in coeff_cases():
+        ref = oracle.solve_batch(oracle.quadratic_errors(c, times.shape[1]), times, B, threads=CORES)
+        plan = binding.Plan(times, B, device=0, table_format=fmt)
+        p, cost, t = binding.solve_batch_coeffs(plan, torch.from_numpy(c).cuda())
+        torch.cuda.synchronize()
+        plan.check_status()
+        assert_same((p.cpu().numpy(), cost.cpu().numpy(), t.cpu().numpy()), ref)
+        # the table route through the library gives the same bits
+        e = binding.quadratic_errors(torch.from_numpy(c).cuda(), times.shape[1])
+        p2, c2, t2 = binding.solve_batch(plan, e)
+        torch.cuda.synchronize()
+        assert_same((p2.cpu().numpy(), c2.cpu().numpy(), t2.cpu().numpy()), ref)
+        plan.close()
+
+
+def test_coefficient_input_host_buffers_cluster_and_tiny_shapes():
+    import torch
+
+    times, B, c = next(coeff_cases())
+    ref = oracle.solve_batch(oracle.quadratic_errors(c, times.shape[1]), times, B, threads=CORES)
+    plan = binding.Plan(times, B, device=0)
+    assert_same(binding.solve_batch_coeffs_host(plan, c), ref)
+    assert_same(binding.solve_batch_coeffs_host(plan, torch.from_numpy(c).pin_memory()), ref)
+    plan.close()
+    for cluster in (2, 8):
+        plan = binding.Plan(times, B, device=0, cluster=cluster)
+        p, cost, t = binding.solve_batch_coeffs(plan, torch.from_numpy(c[:6]).cuda())
+        torch.cuda.synchronize()
+        assert_same((p.cpu().numpy(), cost.cpu().numpy(), t.cpu().numpy()), tuple(x[:6] for x in ref))
+        plan.close()
+    rng = np.random.default_rng(8)
+    for seed in range(60):  # ties, zero and repeated times, K = 1, infeasible budgets
+        wl = W.tiny_random_instance(seed, N=1)
+        c = rng.choice(np.array([0.0, 0.25, 0.5, 1.0], np.float32), size=(5, wl.L)).astype(np.float32)
+        ref = oracle.solve_batch(oracle.quadratic_errors(c, wl.K), wl.times, wl.B)
+        plan = binding.Plan(wl.times, wl.B, device=0)
+        p, cost, t = binding.solve_batch_coeffs(plan, torch.from_numpy(c).cuda())
+        torch.cuda.synchronize()
+        assert_same((p.cpu().numpy(), cost.cpu().numpy(), t.cpu().numpy()), ref)
+        plan.close()
+    with pytest.raises(ValueError):
+        binding.solve_batch_coeffs(binding.Plan(times, B, device=0), torch.zeros((2, 3), device="cuda"))
