@@ -48,6 +48,7 @@ def parse_args():
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--mode", type=int, default=0, help="forward kernel variant (see spdy_options.forward_mode)")
     ap.add_argument("--cluster", type=int, default=0, help="CTAs per candidate (0 = plan's choice)")
+    ap.add_argument("--rows-in-global", type=int, default=0, help="1: row buffers in the workspace (wide-band fallback)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU work budget of the oracle legs")
@@ -214,7 +215,7 @@ def run_ours(args):
     if args.mode:
         fmt = 1 if args.mode in (1, 2) else 2
     plan = binding.Plan(wl.times, wl.B, device=local_rank, table_format=fmt, threads=args.threads,
-                        forward_mode=args.mode, cluster=args.cluster)
+                        forward_mode=args.mode, cluster=args.cluster, rows_in_global=args.rows_in_global)
     info = plan.info
     plan.enable_timing(True)
 

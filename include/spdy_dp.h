@@ -71,7 +71,11 @@ typedef struct spdy_options {
                               identical results, for measurement: 1 compare+select (ARG_U8),
                               2 compare+predicated moves (ARG_U8), 3 fp32 minimum (ROW_F32),
                               4 packed adds + 3-input minimum over choice pairs (ROW_F32) */
-    int32_t reserved[4];   /* must be 0 */
+    int32_t rows_in_global; /* 1: keep the two dynamic-program rows in the workspace (global memory) rather than
+                              in shared memory.  Chosen automatically when a band is too wide even for a
+                              cluster of 8 CTAs (B beyond a few 10^5 buckets); slower, but any width runs.
+                              One CTA of 1024 threads per candidate; not combinable with cluster > 1 */
+    int32_t reserved[3];   /* must be 0 */
 } spdy_options;
 
 /* Facts about a plan: shapes, the launch shape chosen, and work counts for measurement. */
@@ -85,9 +89,9 @@ typedef struct spdy_plan_info {
     int32_t table_format;   /* resolved spdy_table_format */
     int32_t ctas_per_sm;    /* resident CTAs per SM the launch shape allows */
     int32_t sm_count;
-    int32_t reserved0;
+    int32_t rows_in_global; /* 1 if the row buffers live in the workspace */
     int64_t smem_bytes;     /* dynamic shared memory per CTA */
-    int64_t table_bytes_per_candidate; /* walk-back table bytes one candidate needs */
+    int64_t table_bytes_per_candidate; /* workspace one candidate needs: walk-back table (+ row buffers) */
     int64_t band_cells;     /* sum over layers of the live band width (cells written per candidate) */
     int64_t useful_updates; /* sum over (layer, choice) of cells whose source lies in the previous band */
     int64_t issued_updates; /* cell updates the kernel actually issues per candidate (span granularity) */

@@ -30,7 +30,7 @@ EXPORTS = (
 class SpdyOptions(ctypes.Structure):
     _fields_ = [("table_format", ctypes.c_int32), ("threads", ctypes.c_int32),
                 ("cluster", ctypes.c_int32), ("forward_mode", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 4)]
+                ("rows_in_global", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
 
 
 class SpdyPlanInfo(ctypes.Structure):
@@ -38,14 +38,14 @@ class SpdyPlanInfo(ctypes.Structure):
                 ("feasible", ctypes.c_int32), ("max_width", ctypes.c_int32),
                 ("span", ctypes.c_int32), ("threads", ctypes.c_int32), ("cluster", ctypes.c_int32),
                 ("table_format", ctypes.c_int32), ("ctas_per_sm", ctypes.c_int32),
-                ("sm_count", ctypes.c_int32), ("reserved0", ctypes.c_int32),
+                ("sm_count", ctypes.c_int32), ("rows_in_global", ctypes.c_int32),
                 ("smem_bytes", ctypes.c_int64), ("table_bytes_per_candidate", ctypes.c_int64),
                 ("band_cells", ctypes.c_int64), ("useful_updates", ctypes.c_int64),
                 ("issued_updates", ctypes.c_int64), ("nominal_updates", ctypes.c_int64),
                 ("distinct_updates", ctypes.c_int64)]
 
     def as_dict(self) -> dict:
-        return {name: int(getattr(self, name)) for name, _ in self._fields_ if name != "reserved0"}
+        return {name: int(getattr(self, name)) for name, _ in self._fields_}
 
 
 class SpdyError(RuntimeError):
@@ -138,14 +138,14 @@ class Plan:
     """``spdy_plan``: everything that depends only on ``times`` and ``B``."""
 
     def __init__(self, times, B: int, device: int = 0, table_format: int = SPDY_TABLE_DEFAULT,
-                 threads: int = 0, cluster: int = 0, forward_mode: int = 0):
+                 threads: int = 0, cluster: int = 0, forward_mode: int = 0, rows_in_global: int = 0):
         lib = _load()
         t = np.ascontiguousarray(np.asarray(times), dtype=np.int32)
         if t.ndim != 2:
             raise ValueError("times must be [L][K]")
         self.L, self.K, self.B, self.device = int(t.shape[0]), int(t.shape[1]), int(B), int(device)
         opts = SpdyOptions(table_format=table_format, threads=threads, cluster=cluster,
-                           forward_mode=forward_mode)
+                           forward_mode=forward_mode, rows_in_global=rows_in_global)
         handle = ctypes.c_void_p()
         _check(lib.spdy_plan_create(ctypes.byref(handle), t.ctypes.data_as(ctypes.c_void_p),
                                     self.L, self.K, self.B, self.device, ctypes.byref(opts)),

@@ -98,6 +98,7 @@ struct FwdArgs {
     int32_t L, K;
     int32_t row_stride;       // floats per shared-memory row buffer
     int32_t pad;              // +inf guard cells on either side of a row: 32 * the largest cells-per-lane
+    float *grows;             // row buffers in global memory (GROWS kernels), else null
 };
 
 __device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
@@ -358,13 +359,25 @@ __device__ __forceinline__ void process_span(const float *__restrict__ prev, flo
 // RCAP: the largest cells-per-lane this instantiation can run.  The registers a kernel needs grow
 // with the largest unrolled pass, so plans whose rows are narrow (few cells per lane) use the
 // RCAP = 8 build, which fits twice as many CTAs per SM.
-template <int MODE, int NT, int MINB, int RCAP>
+//
+// GROWS: keep the two row buffers in global memory (args.grows, 2 * row_stride floats per candidate of
+// the wave) instead of shared memory.  This is the fallback for bands too wide even for a cluster of
+// eight CTAs; the code is the same, the reads then go through L1/L2.  Writes of one layer are ordered
+// before the reads of the next by the same per-layer __syncthreads().
+template <int MODE, int NT, int MINB, int RCAP, bool GROWS>
 __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs args)
 {
     constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float *rows = reinterpret_cast<float *>(smem_raw);
-    int2 *tap_buf = reinterpret_cast<int2 *>(rows + 2 * static_cast<size_t>(args.row_stride));
+    float *rows;
+    int2 *tap_buf;
+    if constexpr (GROWS) {
+        rows = args.grows + static_cast<size_t>(blockIdx.x) * 2 * static_cast<size_t>(args.row_stride);
+        tap_buf = reinterpret_cast<int2 *>(smem_raw);
+    } else {
+        rows = reinterpret_cast<float *>(smem_raw);
+        tap_buf = reinterpret_cast<int2 *>(rows + 2 * static_cast<size_t>(args.row_stride));
+    }
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -831,7 +844,7 @@ struct FwdVariant {
 };
 
 #define SPDY_VARIANT(MODE, NT, MINB, RCAP) \
-    FwdVariant { MODE, NT, RCAP, spdy_forward_kernel<MODE, NT, MINB, RCAP> }
+    FwdVariant { MODE, NT, RCAP, spdy_forward_kernel<MODE, NT, MINB, RCAP, false> }
 #define SPDY_VARIANTS(MODE)                                                                        \
     SPDY_VARIANT(MODE, 128, 4, RMAX), SPDY_VARIANT(MODE, 256, 2, RMAX), SPDY_VARIANT(MODE, 512, 1, RMAX), \
     SPDY_VARIANT(MODE, 1024, 1, 16), SPDY_VARIANT(MODE, 128, 6, 8), SPDY_VARIANT(MODE, 256, 3, 8),       \
@@ -839,6 +852,13 @@ struct FwdVariant {
 
 const FwdVariant kVariants[] = {
     SPDY_VARIANTS(MODE_ARG), SPDY_VARIANTS(MODE_ARG_PRED), SPDY_VARIANTS(MODE_ROW), SPDY_VARIANTS(MODE_ROW2),
+};
+
+// Rows in global memory: one CTA of 1024 threads per candidate, the default cell update of each
+// table format.
+const FwdVariant kGlobalRowVariants[] = {
+    FwdVariant{MODE_ARG_PRED, 1024, 16, spdy_forward_kernel<MODE_ARG_PRED, 1024, 1, 16, true>},
+    FwdVariant{MODE_ROW2, 1024, 16, spdy_forward_kernel<MODE_ROW2, 1024, 1, 16, true>},
 };
 
 using ClusterKernel = void (*)(const ClusterArgs);
@@ -896,6 +916,7 @@ struct spdy_plan {
     int sm_count = 148;
     int64_t smem_bytes = 0;
     int32_t row_stride = 0, pad = 0;
+    bool global_rows = false;  // row buffers live in the workspace, not in shared memory
     int64_t pitch = 0;  // table cells per candidate
     int64_t band_cells = 0, useful_updates = 0, distinct_updates = 0, issued_updates = 0;
     int32_t max_width = 0;
@@ -947,6 +968,11 @@ void fill_qtab(spdy_plan *p)
 }
 
 int64_t cell_bytes(const spdy_plan *p) { return p->table_format == SPDY_TABLE_ROW_F32 ? 4 : 1; }
+
+// Workspace one candidate needs: its walk-back table, and its two row buffers when those live in
+// global memory.  Both are multiples of 256 bytes.
+int64_t table_bytes_one(const spdy_plan *p) { return std::max<int64_t>(256, round_up(p->pitch * cell_bytes(p), 256)); }
+int64_t row_bytes_one(const spdy_plan *p) { return p->global_rows ? round_up(2LL * p->row_stride * 4, 256) : 0; }
 
 // Live band of every row and the range of every (layer, choice) pair.
 //   lo_l = sum_{j<=l} mn_j,  hi_l = min(B, sum_{j<=l} mx_j, B - sum_{j>l} mn_j)
@@ -1239,6 +1265,28 @@ int choose_cluster_shape(spdy_plan *p, const spdy_options *opts, int64_t smem_pe
     return requested ? SPDY_ERR_INVALID_ARG : SPDY_ERR_UNSUPPORTED;
 }
 
+// Wide-band fallback: one CTA of 1024 threads per candidate, row buffers in the workspace.
+int choose_global_row_shape(spdy_plan *p)
+{
+    const int threads = 1024;
+    if (threads < p->K) return SPDY_ERR_UNSUPPORTED;
+    p->mode = p->table_format == SPDY_TABLE_ARG_U8 ? MODE_ARG_PRED : MODE_ROW2;
+    p->cluster = 1;
+    p->cvariant = nullptr;
+    p->slices.clear();
+    int rc = layout_table(p, threads, nullptr);
+    if (rc != SPDY_OK) return rc;
+    p->global_rows = true;
+    p->smem_bytes = 2LL * ((p->K + 1) & ~1) * 8;
+    p->threads = threads;
+    p->variant = nullptr;
+    for (const FwdVariant &v : kGlobalRowVariants)
+        if (v.mode == p->mode) p->variant = &v;
+    if (!p->variant) return SPDY_ERR_INVALID_ARG;
+    p->ctas_per_sm = 1;
+    return SPDY_OK;
+}
+
 int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
 {
     int64_t smem_per_sm = 233472, smem_per_block = 232448;
@@ -1268,6 +1316,12 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
     if (opts && opts->cluster != 0 && opts->cluster != 1 && opts->cluster != 2 && opts->cluster != 4 &&
         opts->cluster != 8)
         return SPDY_ERR_INVALID_ARG;
+    p->global_rows = false;
+    if (opts && opts->rows_in_global != 0 && opts->rows_in_global != 1) return SPDY_ERR_INVALID_ARG;
+    if (opts && opts->rows_in_global) {
+        if (opts->cluster > 1) return SPDY_ERR_INVALID_ARG;
+        return choose_global_row_shape(p);
+    }
     if (opts && opts->cluster > 1) return choose_cluster_shape(p, opts, smem_per_block);
 
     // Candidate CTA sizes; keep the one whose rounds are fullest, preferring more resident warps.
@@ -1292,10 +1346,15 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
         }
     }
     if (best_threads == 0) {
-        // No single CTA can hold two rows of this width: split each candidate over a cluster,
-        // unless the caller insisted on one CTA.
+        // No single CTA can hold two rows of this width in shared memory (the caller may have
+        // insisted on that).
         if (opts && opts->cluster == 1) return SPDY_ERR_UNSUPPORTED;
-        return choose_cluster_shape(p, opts, smem_per_block);
+        // Rows in global memory, read through L1, measured faster than a cluster for such widths
+        // (B = 10^5: 1.6x, B = 2*10^5: 1.9x) and have no width limit.  A cluster is still used when the
+        // caller asks for one (cluster > 1, handled above) or pins a launch shape the fallback lacks.
+        if (opts && ((opts->threads && opts->threads != 1024) || opts->forward_mode))
+            return choose_cluster_shape(p, opts, smem_per_block);
+        return choose_global_row_shape(p);
     }
     int rc = layout_table(p, best_threads, nullptr);
     if (rc != SPDY_OK) return rc;
@@ -1442,7 +1501,7 @@ int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int3
     *out = nullptr;
     if (!times_host || L < 1 || K < 1 || K > 255 || B < 0 || device < -1) return SPDY_ERR_INVALID_ARG;
     if (opts) {
-        for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < 3; ++i)
             if (opts->reserved[i] != 0) return SPDY_ERR_INVALID_ARG;
         if (opts->threads != 0 && (opts->threads % 32 != 0 || opts->threads < 32 || opts->threads > 1024))
             return SPDY_ERR_INVALID_ARG;
@@ -1501,6 +1560,7 @@ int spdy_plan_get_info(const spdy_plan *plan, spdy_plan_info *info)
     info->table_format = plan->table_format;
     info->ctas_per_sm = plan->ctas_per_sm;
     info->sm_count = plan->sm_count;
+    info->rows_in_global = plan->global_rows ? 1 : 0;
     info->smem_bytes = plan->smem_bytes;
     info->table_bytes_per_candidate = static_cast<int64_t>(spdy_workspace_bytes(plan, 1));
     info->band_cells = plan->band_cells;
@@ -1524,8 +1584,7 @@ int spdy_plan_get_bands(const spdy_plan *plan, int32_t *lo_host, int32_t *width_
 size_t spdy_workspace_bytes(const spdy_plan *plan, int64_t N)
 {
     if (!plan || N <= 0) return 0;
-    const int64_t per = std::max<int64_t>(256, round_up(plan->pitch * cell_bytes(plan), 256));
-    return static_cast<size_t>(per) * static_cast<size_t>(N);
+    return static_cast<size_t>(table_bytes_one(plan) + row_bytes_one(plan)) * static_cast<size_t>(N);
 }
 
 }  // extern "C"
@@ -1557,9 +1616,12 @@ int solve_impl(const spdy_plan *plan, const float *errors_dev, const float *coef
     const size_t per = spdy_workspace_bytes(plan, 1);
     const int64_t wave = static_cast<int64_t>(std::min<size_t>(workspace_bytes / per, static_cast<size_t>(N)));
     if (wave < 1) return SPDY_ERR_WORKSPACE_TOO_SMALL;
-    // The table pitch handed to the kernels is in cells; `per` bytes per candidate keeps every
-    // candidate's table 256-byte aligned.
-    const int64_t pitch_cells = static_cast<int64_t>(per) / cell_bytes(plan);
+    // The table pitch handed to the kernels is in cells; every candidate's table is 256-byte aligned.
+    const int64_t pitch_cells = table_bytes_one(plan) / cell_bytes(plan);
+    // Row buffers in global memory (wide-band fallback) follow the tables of the wave.
+    float *grows = plan->global_rows
+                       ? reinterpret_cast<float *>(static_cast<unsigned char *>(workspace_dev) + wave * table_bytes_one(plan))
+                       : nullptr;
 
     spdy_plan *mplan = const_cast<spdy_plan *>(plan);  // timing state only
     if (plan->timing) mplan->events_used = 0;
@@ -1595,6 +1657,7 @@ int solve_impl(const spdy_plan *plan, const float *errors_dev, const float *coef
         fa.K = plan->K;
         fa.row_stride = plan->row_stride;
         fa.pad = plan->pad;
+        fa.grows = grows;
         // Grid x is limited to 2^31-1 CTAs, far above any wave that fits in memory.
         if (plan->cluster > 1) {
             ClusterArgs ca;

@@ -214,13 +214,20 @@ def test_cluster_split_of_one_candidate_gives_the_same_answer(cluster, mode):
 
 
 @pytest.mark.parametrize("fmt", FORMATS)
-def test_budget_100000_needs_a_cluster(fmt):
-    """B = 100000: a band-limited row is about 210 KB, so two rows cannot live in one CTA."""
+def test_budget_100000_does_not_fit_one_cta(fmt):
+    """B = 100000: a band-limited row is about 210 KB, so two rows cannot live in one CTA's shared
+    memory.  By default the rows then go to global memory; on request a cluster shares them."""
     wl = W.make_workload(4, N=5, B=100000)
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
     plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
-    assert plan.info["cluster"] > 1
+    assert plan.info["rows_in_global"] == 1 and plan.info["cluster"] == 1
     plan.close()
-    assert_same(gpu_solve(wl, fmt), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+    assert_same(gpu_solve(wl, fmt), ref)
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt, cluster=4)
+    assert plan.info["cluster"] == 4 and plan.info["rows_in_global"] == 0
+    plan.close()
+    assert_same(gpu_solve(wl, fmt, cluster=4), ref)
+    assert_same(gpu_solve(wl, fmt, threads=512), ref)  # a pinned CTA size selects the cluster path
 
 
 def test_cluster_with_ties_and_wide_rows():
@@ -308,3 +315,37 @@ def test_coefficient_input_host_buffers_cluster_and_tiny_shapes():
         plan.close()
     with pytest.raises(ValueError):
         binding.solve_batch_coeffs(binding.Plan(times, B, device=0), torch.zeros((2, 3), device="cuda"))
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_rows_in_global_memory_give_the_same_answer(fmt):
+    """The wide-band fallback (row buffers in the workspace instead of shared memory), forced on
+    shapes the oracle finishes quickly."""
+    import torch
+
+    wl = W.make_workload(2, N=7)
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+    assert_same(gpu_solve(wl, fmt, rows_in_global=1), ref)
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt, rows_in_global=1)
+    assert plan.info["rows_in_global"] == 1 and plan.info["threads"] == 1024
+    ws = torch.empty(plan.workspace_bytes(3), dtype=torch.uint8, device="cuda")  # 7 candidates in 3 waves
+    p, c, t = binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda(), workspace=ws)
+    torch.cuda.synchronize()
+    plan.check_status()
+    assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), ref)
+    plan.close()
+    for seed in range(40):
+        for exact in (False, True):
+            tiny = W.tiny_random_instance(seed + (10_000 if exact else 0), exact=exact, N=4)
+            assert_same(gpu_solve(tiny, fmt, rows_in_global=1), oracle.solve_batch(tiny.errors, tiny.times, tiny.B))
+    with pytest.raises(binding.SpdyError):
+        binding.Plan(wl.times, wl.B, device=0, rows_in_global=1, cluster=2)
+
+
+def test_budget_400000_falls_back_to_rows_in_global_memory():
+    """B = 400000: a band of about 210 000 cells does not fit a cluster of eight CTAs either."""
+    wl = W.make_workload(4, N=2, B=400000)
+    plan = binding.Plan(wl.times, wl.B, device=0)
+    assert plan.info["rows_in_global"] == 1 and plan.info["cluster"] == 1
+    plan.close()
+    assert_same(gpu_solve(wl), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))

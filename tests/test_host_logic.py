@@ -146,10 +146,15 @@ def test_infeasible_and_degenerate_plans():
     assert binding.Plan(over, 10, device=-1).info["feasible"] == 0
 
 
-def test_wide_rows_choose_a_cluster():
+def test_wide_rows_leave_shared_memory():
     wl = W.make_workload(4, N=1, B=100000)
     info = binding.Plan(wl.times, wl.B, device=-1).info
-    assert info["cluster"] in (2, 4, 8) and info["smem_bytes"] <= 232448
+    assert info["rows_in_global"] == 1 and info["cluster"] == 1 and info["threads"] == 1024
+    info = binding.Plan(wl.times, wl.B, device=-1, threads=512).info
+    assert info["cluster"] in (2, 4, 8) and info["smem_bytes"] <= 232448 and info["rows_in_global"] == 0
+    for c in (4, 8):
+        info = binding.Plan(wl.times, wl.B, device=-1, cluster=c).info
+        assert info["cluster"] == c and info["smem_bytes"] <= 232448
     with pytest.raises(binding.SpdyError) as e:  # one CTA cannot hold it
         binding.Plan(wl.times, wl.B, device=-1, cluster=1)
     assert e.value.status == -3
