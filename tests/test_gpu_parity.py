@@ -170,6 +170,48 @@ def test_host_buffer_and_one_shot_entry_points():
     assert (p.cpu().numpy() == 0xFF).all() and (t.cpu().numpy() == -1).all() and np.isposinf(c.cpu().numpy()).all()
 
 
+def check_full_size(wl, sample_size, fmt=0, workspace_bytes=None):
+    """Invariants that hold at any size on every candidate, and the oracle on a seeded sample."""
+    import torch
+
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+    ws = None
+    if workspace_bytes is not None:
+        per = plan.workspace_bytes(1)
+        ws = torch.empty(max(per, workspace_bytes // per * per), dtype=torch.uint8, device="cuda")
+    p, c, t = binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda(), workspace=ws)
+    torch.cuda.synchronize()
+    plan.check_status()
+    p, c, t = p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()
+    del ws
+    plan.close()
+    assert (t >= 0).all() and (t <= wl.B).all() and (p < wl.K).all()
+    idx = p.astype(np.int64)
+    assert np.array_equal(wl.times[np.arange(wl.L)[None, :], idx].sum(axis=1), t)
+    e_sel = np.take_along_axis(wl.errors, idx[:, :, None], axis=2)[:, :, 0]
+    acc = np.zeros(wl.N, np.float32)
+    for l in range(wl.L):
+        acc = (acc + e_sel[:, l]).astype(np.float32)
+    assert acc.tobytes() == c.tobytes()
+    sample = np.sort(np.random.default_rng(0).choice(wl.N, size=min(sample_size, wl.N), replace=False))
+    ref = oracle.solve_batch(wl.errors[sample], wl.times, wl.B, threads=CORES)
+    assert_same((p[sample], c[sample], t[sample]), ref)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_full_size_resnet50_and_bert_large_batches(fmt):
+    """Configs 1 and 3 at their full N = 1024, in the launch shape the plan picks by default."""
+    check_full_size(W.make_workload(1), 96, fmt)
+    check_full_size(W.make_workload(3), 8, fmt)
+
+
+def test_full_size_sweep_points():
+    """Config 4's largest points: N = 65536 (run in waves inside a 12 GB workspace) and B = 100000."""
+    check_full_size(W.make_workload(4, N=65536), 64, workspace_bytes=12 << 30)
+    check_full_size(W.make_workload(4, N=4096, B=1000), 256)
+    check_full_size(W.make_workload(4, N=1024, B=100000), 6)
+
+
 def test_full_size_bert_base_batch_in_the_benchmark_configuration():
     """N = 4096 as the benchmark times it: invariants on every candidate, oracle on a sample."""
     import torch
