@@ -31,8 +31,8 @@ CELLS_PER_CLK_PER_SM = 32.0  # one 4-byte shared-memory read per cell update, 32
 # DRAM bytes (read + write) of the forward kernel per candidate from an ncu capture of one wave
 # (592 candidates) of the BERT-base shape; traffic grows in proportion to N.  Valid only for the
 # library version the counters were taken with.
-NCU_TRAFFIC = {"version": 1001, "workload_prefix": "bert-base-L72-K42-B10000",
-               "bytes_per_candidate": {"row_f32": 764.2e6 / 592, "arg_u8": 157.0e6 / 592}}
+NCU_TRAFFIC = {"version": 1003, "workload_prefix": "bert-base-L72-K42-B10000",
+               "bytes_per_candidate": {"row_f32": 762.88e6 / 592, "arg_u8": 153.30e6 / 592}}
 
 
 def parse_args():
@@ -286,6 +286,25 @@ def run_ours(args):
                "h2d_bytes_per_step": int(h_err.numel() * 4),
                "d2h_bytes_per_step": int(wl.N * (wl.L + 8)), "ms_per_step": 1e3 * e2e_s / args.steps}
 
+    # The same end-to-end step with Eq. 4's coefficients as input (what one search step submits):
+    # K times fewer bytes go to the device.  Extra figure; the headline `e2e` above takes error tables.
+    e2e_coeffs = None
+    if not args.no_e2e:
+        h_c = torch.from_numpy(W.sensitivity_samples(7000 + rank, wl.L, wl.N)).pin_memory()
+        for _ in range(2):
+            binding.solve_batch_coeffs_host(plan, h_c, h_prof, h_cost, h_time, stream)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            binding.solve_batch_coeffs_host(plan, h_c, h_prof, h_cost, h_time, stream)
+        torch.cuda.synchronize()
+        c_s = sharding.max_over_ranks(time.perf_counter() - t0, dev)
+        plan.check_status()
+        e2e_coeffs = {"value": sharding.whole_job_rate(wl.N * args.steps, world, c_s), "unit": "candidates/s",
+                      "h2d_bytes_per_step": int(h_c.numel() * 4), "d2h_bytes_per_step": int(wl.N * (wl.L + 8)),
+                      "ms_per_step": 1e3 * c_s / args.steps,
+                      "input": "Eq. 4 coefficients [N][L], uniform in [0,1] (spdy_solve_batch_coeffs_host)"}
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -348,6 +367,8 @@ def run_ours(args):
     }
     if e2e:
         line["e2e"] = e2e
+    if e2e_coeffs:
+        line["e2e_coeffs"] = e2e_coeffs
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = oracle_baseline(wl, args.cpu_seconds)
     print(json.dumps(line), flush=True)
