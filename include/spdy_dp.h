@@ -151,7 +151,10 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
  * Same computation with HOST buffers (pageable or pinned): copies errors to the device, solves,
  * copies the three outputs back and waits for the stream.  Device staging memory is owned by
  * the plan and grows on demand (cudaMalloc on first use or growth), so one plan must not run
- * two host-buffer solves at the same time.
+ * two host-buffer solves at the same time.  An error table larger than one wave of CTAs is uploaded in
+ * a few chunks on a second, plan-owned stream (ordered after the work already queued on `cuda_stream`),
+ * each chunk's kernels waiting only for their own chunk, so that with pinned host memory the upload
+ * hides behind the kernels.
  */
 int spdy_solve_batch_host(spdy_plan *plan, const float *errors_host, int64_t N,
                           uint8_t *profile_host, float *cost_host, int32_t *time_used_host,

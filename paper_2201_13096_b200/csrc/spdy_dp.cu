@@ -950,6 +950,11 @@ struct spdy_plan {
     bool timing = false;
     std::vector<cudaEvent_t> events;
     size_t events_used = 0;
+    // host-buffer entry points: a second stream and events that let the upload of one chunk of
+    // candidates overlap the kernels of the chunk before it
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t entry_event = nullptr;
+    std::vector<cudaEvent_t> copy_events;
     // staging for the host-buffer entry point
     unsigned char *d_arena = nullptr;
     size_t arena_bytes = 0;
@@ -1541,6 +1546,9 @@ void spdy_plan_destroy(spdy_plan *plan)
         if (plan->d_blob) cudaFree(plan->d_blob);
         if (plan->d_arena) cudaFree(plan->d_arena);
         for (cudaEvent_t e : plan->events) cudaEventDestroy(e);
+        for (cudaEvent_t e : plan->copy_events) cudaEventDestroy(e);
+        if (plan->entry_event) cudaEventDestroy(plan->entry_event);
+        if (plan->copy_stream) cudaStreamDestroy(plan->copy_stream);
     }
     delete plan;
 }
@@ -1594,7 +1602,7 @@ namespace {
 // The whole path for one batch; exactly one of errors_dev / coeffs_dev is non-null.
 int solve_impl(const spdy_plan *plan, const float *errors_dev, const float *coeffs_dev, int64_t N,
                uint8_t *profile_dev, float *cost_dev, int32_t *time_used_dev, void *workspace_dev,
-               size_t workspace_bytes, void *cuda_stream)
+               size_t workspace_bytes, void *cuda_stream, bool keep_timing = false)
 {
     if (!plan || plan->device < 0 || N < 0) return SPDY_ERR_INVALID_ARG;
     if (N == 0) return SPDY_OK;
@@ -1624,7 +1632,7 @@ int solve_impl(const spdy_plan *plan, const float *errors_dev, const float *coef
                        : nullptr;
 
     spdy_plan *mplan = const_cast<spdy_plan *>(plan);  // timing state only
-    if (plan->timing) mplan->events_used = 0;
+    if (plan->timing && !keep_timing) mplan->events_used = 0;
     for (int64_t first = 0; first < N; first += wave) {
         const int64_t count = std::min<int64_t>(wave, N - first);
         cudaEvent_t *ev = nullptr;
@@ -1830,10 +1838,54 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
     uint8_t *d_profile = base + off_profile;
     float *d_cost = reinterpret_cast<float *>(base + off_cost);
     int32_t *d_time = reinterpret_cast<int32_t *>(base + off_time);
-    SPDY_CUDA_TRY(cudaMemcpyAsync(d_err, errors_host, err_bytes, cudaMemcpyHostToDevice, stream));
-    rc = solve_impl(plan, coeffs ? nullptr : d_err, coeffs ? d_err : nullptr, N, d_profile, d_cost, d_time,
-                    base + off_ws, ws_bytes, stream);
-    if (rc != SPDY_OK) return rc;
+    // An error table goes up in chunks of growing size (one full wave of CTAs first, then six times
+    // the previous chunk) on a second stream, so that every upload but the first hides behind the
+    // kernels of the chunk before it; an upload takes about a seventh of the time its candidates take
+    // to solve.  Every chunk costs one more latency-bound walk-back launch, so chunks are few, and
+    // coefficient input (K times smaller) goes up in one piece.
+    const int64_t per_cand = static_cast<int64_t>(plan->L) * (coeffs ? 1 : plan->K);
+    std::vector<int64_t> bounds(1, 0);
+    {
+        int64_t size = std::max<int64_t>(1, static_cast<int64_t>(plan->ctas_per_sm) * plan->sm_count / std::max(1, plan->cluster));
+        if (coeffs) size = N;
+        while (bounds.back() < N) {
+            bounds.push_back(std::min<int64_t>(N, bounds.back() + size));
+            size *= 6;
+        }
+    }
+    const size_t chunks = bounds.size() - 1;
+    if (chunks > 1) {
+        if (!plan->copy_stream) SPDY_CUDA_TRY(cudaStreamCreateWithFlags(&plan->copy_stream, cudaStreamNonBlocking));
+        if (!plan->entry_event) SPDY_CUDA_TRY(cudaEventCreateWithFlags(&plan->entry_event, cudaEventDisableTiming));
+        while (plan->copy_events.size() < chunks) {
+            cudaEvent_t e;
+            SPDY_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+            plan->copy_events.push_back(e);
+        }
+        // Work already queued on the caller's stream may still read the staging buffer.
+        SPDY_CUDA_TRY(cudaEventRecord(plan->entry_event, stream));
+        SPDY_CUDA_TRY(cudaStreamWaitEvent(plan->copy_stream, plan->entry_event, 0));
+        for (size_t c = 0; c < chunks; ++c) {
+            const int64_t first = bounds[c], count = bounds[c + 1] - bounds[c];
+            SPDY_CUDA_TRY(cudaMemcpyAsync(d_err + first * per_cand, errors_host + first * per_cand,
+                                          static_cast<size_t>(count * per_cand) * sizeof(float),
+                                          cudaMemcpyHostToDevice, plan->copy_stream));
+            SPDY_CUDA_TRY(cudaEventRecord(plan->copy_events[c], plan->copy_stream));
+        }
+    } else {
+        SPDY_CUDA_TRY(cudaMemcpyAsync(d_err, errors_host, err_bytes, cudaMemcpyHostToDevice, stream));
+    }
+    for (size_t c = 0; c < chunks; ++c) {
+        const int64_t first = bounds[c], count = bounds[c + 1] - bounds[c];
+        if (chunks > 1) SPDY_CUDA_TRY(cudaStreamWaitEvent(stream, plan->copy_events[c], 0));
+        const float *in = d_err + first * per_cand;
+        rc = solve_impl(plan, coeffs ? nullptr : in, coeffs ? in : nullptr, count, d_profile + first * plan->L,
+                        d_cost + first, d_time + first, base + off_ws, ws_bytes, stream, c > 0);
+        if (rc != SPDY_OK) {
+            if (chunks > 1) cudaStreamSynchronize(plan->copy_stream);
+            return rc;
+        }
+    }
     SPDY_CUDA_TRY(cudaMemcpyAsync(profile_host, d_profile, static_cast<size_t>(N) * plan->L, cudaMemcpyDeviceToHost, stream));
     SPDY_CUDA_TRY(cudaMemcpyAsync(cost_host, d_cost, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
     SPDY_CUDA_TRY(cudaMemcpyAsync(time_used_host, d_time, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));

@@ -391,3 +391,32 @@ def test_budget_400000_falls_back_to_rows_in_global_memory():
     assert plan.info["rows_in_global"] == 1 and plan.info["cluster"] == 1
     plan.close()
     assert_same(gpu_solve(wl), oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
+
+
+def test_host_buffer_path_uploads_in_chunks():
+    """Batches larger than one wave go up in several chunks on a second stream; results must not
+    depend on that, call after call, for error tables and for coefficients."""
+    import torch
+
+    wl = W.make_workload(1, N=2500)
+    plan = binding.Plan(wl.times, wl.B, device=0)
+    p, c, t = binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda())
+    torch.cuda.synchronize()
+    dev = (p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy())
+    pinned = torch.from_numpy(wl.errors).pin_memory()
+    for errors in (wl.errors, pinned, wl.errors[:700], wl.errors):
+        n = len(errors)
+        assert_same(binding.solve_batch_host(plan, errors), tuple(x[:n] for x in dev))
+    sample = np.arange(0, 2500, 97)
+    assert_same(tuple(x[sample] for x in dev), oracle.solve_batch(wl.errors[sample], wl.times, wl.B, threads=CORES))
+    coeffs = W.sensitivity_samples(3, wl.L, 2500)
+    pc, cc, tc = binding.solve_batch_coeffs(plan, torch.from_numpy(coeffs).cuda())
+    torch.cuda.synchronize()
+    assert_same(binding.solve_batch_coeffs_host(plan, coeffs), (pc.cpu().numpy(), cc.cpu().numpy(), tc.cpu().numpy()))
+    plan.enable_timing(True)  # timing covers all chunks of a host-buffer call
+    binding.solve_batch_host(plan, pinned)
+    fwd_host, _ = plan.last_timing()
+    binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda())
+    fwd_dev, _ = plan.last_timing()
+    assert 0.5 * fwd_dev < fwd_host < 3.0 * fwd_dev
+    plan.close()
