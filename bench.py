@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--mode", type=int, default=0, help="forward kernel variant (see spdy_options.forward_mode)")
     ap.add_argument("--cluster", type=int, default=0, help="CTAs per candidate (0 = plan's choice)")
     ap.add_argument("--rows-in-global", type=int, default=0, help="1: row buffers in the workspace (wide-band fallback)")
+    ap.add_argument("--search", type=int, default=0, metavar="TRIALS",
+                    help="also run Algorithm 4 with this many trials per loop on the workload's timing table "
+                         "(synthetic loss) and report where the time goes, under the key 'search'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU work budget of the oracle legs")
@@ -369,6 +372,22 @@ def run_ours(args):
         line["e2e"] = e2e
     if e2e_coeffs:
         line["e2e_coeffs"] = e2e_coeffs
+    if args.search > 0:
+        from paper_2201_13096_b200 import search as S
+
+        solver = S.gpu_solver(wl.times, wl.B, device=local_rank)
+        loss = W.synthetic_calibration_loss(args.config, wl.L, wl.K)
+        t0 = time.perf_counter()
+        res = S.search(wl.times, wl.B, W.sensitivity_samples(args.config, wl.L, 1)[0],
+                       W.sensitivity_samples(args.config + 100, wl.L, args.search),
+                       W.mutation_draws(args.config, wl.L), loss, trials=args.search, solver=solver)
+        wall = time.perf_counter() - t0
+        line["search"] = {"trials_per_loop": args.search, "neighbourhood_sizes": int(np.ceil(0.1 * wl.L)),
+                          "evals": res["evals"], "accepted": len(res["accepted"]), "loss": res["loss"],
+                          "dp_batches": res["dp_batches"], "dp_candidates": res["dp_candidates"],
+                          "dp_ms": 1e3 * res["dp_seconds"], "eval_ms": 1e3 * res["eval_seconds"], "wall_ms": 1e3 * wall,
+                          "note": "synthetic loss (microseconds per call); with a real stitched-model evaluation "
+                                  "the evaluations dominate, as the paper reports"}
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = oracle_baseline(wl, args.cpu_seconds)
     print(json.dumps(line), flush=True)

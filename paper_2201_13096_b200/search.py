@@ -18,6 +18,7 @@ the caller's: ``eval_fn(profile) -> float``, lower is better, +inf for an infeas
 from __future__ import annotations
 
 import math
+import time
 from typing import Callable, Optional
 
 import numpy as np
@@ -54,25 +55,31 @@ def search(times, B: int, c0, phase1, draws: Callable[[int, int], tuple],
     ``solver`` defaults to the CUDA library on ``device``; there is no CPU implementation here.
 
     Returns a dict: ``c`` [L] fp32, ``profile`` [L] uint8, ``loss``, ``evals`` (calls of ``eval_fn``),
-    ``accepted`` (list of (d, j), d = 0 for the first loop), ``dp_batches``, ``dp_candidates``.
+    ``accepted`` (list of (d, j), d = 0 for the first loop), ``dp_batches``, ``dp_candidates``, and the wall
+    time spent in the solver and in ``eval_fn`` (``dp_seconds``, ``eval_seconds``).
     """
     times = np.ascontiguousarray(np.asarray(times), dtype=np.int32)
     L = int(times.shape[0])
     if solver is None:
         solver = gpu_solver(times, B, device=device)
-    stats = {"evals": 0, "dp_batches": 0, "dp_candidates": 0}
+    stats = {"evals": 0, "dp_batches": 0, "dp_candidates": 0, "dp_seconds": 0.0, "eval_seconds": 0.0}
 
     def solve(coeffs: np.ndarray) -> np.ndarray:
         out = []
+        t0 = time.perf_counter()
         for lo in range(0, len(coeffs), max_batch):
             out.append(np.asarray(solver(coeffs[lo:lo + max_batch])))
             stats["dp_batches"] += 1
         stats["dp_candidates"] += len(coeffs)
+        stats["dp_seconds"] += time.perf_counter() - t0
         return np.concatenate(out, axis=0)
 
     def evaluate(profile: np.ndarray) -> float:
         stats["evals"] += 1
-        return float(eval_fn(profile))
+        t0 = time.perf_counter()
+        value = float(eval_fn(profile))
+        stats["eval_seconds"] += time.perf_counter() - t0
+        return value
 
     c_star = np.array(c0, dtype=np.float32)
     phase1 = np.asarray(phase1, dtype=np.float32)[:trials]
