@@ -322,6 +322,10 @@ def run_ours(args):
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
     except Exception:
         pass
+    try:
+        probe = binding.probe_peaks(local_rank)
+    except binding.SpdyError:
+        probe = (0.0, 0.0)
     sm_max = float(peaks.get("sm_max_mhz", SM_MAX_MHZ_NOMINAL))
     peak_cells = info["sm_count"] * sm_max * 1e6 * CELLS_PER_CLK_PER_SM
     # Work the forward pass has to do per launch: one update per (cell, distinct shift) pair.
@@ -358,6 +362,11 @@ def run_ours(args):
             "traffic_unit": "bytes per launch (ncu dram read+write on one wave, scaled by N)",
             "peak_is": f"{info['sm_count']} SMs x {sm_max:.0f} MHz x 32 four-byte shared-memory reads per clock "
                        "(one read per cell update); of nominal unit counts, max clock of measured",
+            "peak_measured": probe[0] / 1e9, "frac_of_measured": (achieved / probe[0]) if probe[0] else None,
+            "arithmetic_peak_measured": probe[1] / 1e9,
+            "peak_measured_is": "spdy_probe_peaks on this device in this run: lane-consecutive 4-byte shared-memory "
+                                "reads per second (the binding ceiling), and cell updates per second of the "
+                                "arithmetic alone on registers",
             "kernel_ms": fwd, "walkback_ms": back,
             "distinct_updates_per_launch": useful / waves, "issued_updates_per_launch": info["issued_updates"] * wl.N / waves,
         },

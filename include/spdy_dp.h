@@ -275,6 +275,17 @@ int spdy_solve_batch_static(const float *errors_dev, const int32_t *times_host, 
 /* Size in bytes of the array spdy_solve_batch_static works in (SPDY_STATIC_SCRATCH_BYTES). */
 size_t spdy_static_scratch_bytes(void);
 
+/*
+ * Measurement aid: the two ceilings of the forward pass (Eq. 2's update = one read of the previous row,
+ * one add, one minimum) as this device delivers them, from two short probe kernels on the default
+ * stream of `device` (about 50 ms; allocates and frees a small buffer; synchronous).
+ *   *lds_reads_per_s          4-byte shared-memory reads per second, lane-consecutive, all SMs
+ *   *cell_updates_alu_per_s   cell updates per second of the arithmetic alone (packed fp32 adds and
+ *                             3-input minima on registers)
+ * Either pointer may be NULL.  Errors: INVALID_ARG, NO_MEMORY, CUDA.
+ */
+int spdy_probe_peaks(int device, double *lds_reads_per_s, double *cell_updates_alu_per_s);
+
 /* Static, human-readable text for a status code. */
 const char *spdy_strerror(int status);
 

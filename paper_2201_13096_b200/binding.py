@@ -23,7 +23,7 @@ EXPORTS = (
     "spdy_plan_check_status", "spdy_plan_enable_timing", "spdy_plan_last_timing",
     "spdy_solve_batch_static", "spdy_static_scratch_bytes", "spdy_strerror", "spdy_last_cuda_error", "spdy_version",
     "spdy_solve_batch_coeffs", "spdy_solve_batch_coeffs_host", "spdy_quadratic_errors",
-    "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile",
+    "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile", "spdy_probe_peaks",
 )
 
 
@@ -97,6 +97,8 @@ def _load():
     lib.spdy_bucketize_times.argtypes = [vp, i32, i32, ctypes.c_double, i32, i32, vp]
     lib.spdy_uniform_profile.restype = ctypes.c_int
     lib.spdy_uniform_profile.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i64)]
+    lib.spdy_probe_peaks.restype = ctypes.c_int
+    lib.spdy_probe_peaks.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     lib.spdy_solve_batch_simple.restype = ctypes.c_int
     lib.spdy_solve_batch_simple.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.spdy_plan_check_status.restype = ctypes.c_int
@@ -377,3 +379,10 @@ def uniform_profile(times, B: int, keep_dense=None):
                                         None if keep is None else keep.ctypes.data_as(ctypes.c_void_p),
                                         ctypes.byref(k), ctypes.byref(total)), "spdy_uniform_profile")
     return int(k.value), int(total.value)
+
+
+def probe_peaks(device: int = 0):
+    """``spdy_probe_peaks``: (shared-memory 4-byte reads per second, arithmetic-only cell updates per second)."""
+    lds, alu = ctypes.c_double(), ctypes.c_double()
+    _check(_load().spdy_probe_peaks(int(device), ctypes.byref(lds), ctypes.byref(alu)), "spdy_probe_peaks")
+    return float(lds.value), float(alu.value)

@@ -802,6 +802,63 @@ __global__ void spdy_backtrack_row_kernel(const BackArgs args)
     if ((!ok || t != 0) && lane == 0) atomicExch(args.status, 1);
 }
 
+// ----------------------------------------------------------------------------------------------
+// Peak probes: what the forward kernel's two ceilings amount to on the device at hand
+// ----------------------------------------------------------------------------------------------
+//
+// spdy_probe_lds_kernel streams 4-byte shared-memory reads the way the forward kernel issues them
+// (lane-consecutive, a different word offset per read) into running minima; spdy_probe_alu_kernel
+// runs the arithmetic of one cell update (one packed add per two cells, one 3-input minimum per two
+// updates) on registers only.  Each thread reports its result so that nothing is optimised away.
+constexpr int PROBE_WORDS = 8192;  // floats of shared memory a probe CTA reads from
+
+__global__ void __launch_bounds__(256) spdy_probe_lds_kernel(float *out, int iters)
+{
+    __shared__ float buf[PROBE_WORDS + 1024];
+    for (int i = threadIdx.x; i < PROBE_WORDS + 1024; i += blockDim.x) buf[i] = static_cast<float>(i & 1023);
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = pos_inf();
+    int off = warp * 37;
+    for (int it = 0; it < iters; ++it) {
+        const float *src = buf + (off & (PROBE_WORDS - 1)) + lane;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = fminf(acc[j], src[j * 32]);
+        off += 293;  // an odd stride: every read starts at a different bank
+    }
+    float r = acc[0];
+#pragma unroll
+    for (int j = 1; j < 8; ++j) r = fminf(r, acc[j]);
+    out[blockIdx.x * blockDim.x + threadIdx.x] = r;
+}
+
+__global__ void __launch_bounds__(256) spdy_probe_alu_kernel(float *out, int iters, float e0, float e1)
+{
+    float best[8], a[8], b[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        best[j] = pos_inf();
+        a[j] = static_cast<float>(threadIdx.x + j);
+        b[j] = static_cast<float>(threadIdx.x * 3 + j);
+    }
+    const unsigned long long e0s = splat2(e0), e1s = splat2(e1);
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+            add2_rn(a[j], a[j + 1], e0s);
+            add2_rn(b[j], b[j + 1], e1s);
+            best[j] = min3(best[j], a[j], b[j]);
+            best[j + 1] = min3(best[j + 1], a[j + 1], b[j + 1]);
+        }
+    }
+    float r = best[0];
+#pragma unroll
+    for (int j = 1; j < 8; ++j) r = fminf(r, best[j]);
+    out[blockIdx.x * blockDim.x + threadIdx.x] = r;
+}
+
 // Eq. 4 written out as a table: errors[n][l][i] = c[n][l] * (i / (K-1))^2, the same fp32 multiply
 // of the coefficient with the pre-rounded square that the solver's coefficient mode performs in place.
 __global__ void spdy_quadratic_errors_kernel(const float *coeffs, float *errors, int64_t total, int32_t K)
@@ -846,7 +903,7 @@ struct FwdVariant {
 #define SPDY_VARIANT(MODE, NT, MINB, RCAP) \
     FwdVariant { MODE, NT, RCAP, spdy_forward_kernel<MODE, NT, MINB, RCAP, false> }
 #define SPDY_VARIANTS(MODE)                                                                        \
-    SPDY_VARIANT(MODE, 128, 4, RMAX), SPDY_VARIANT(MODE, 256, 2, RMAX), SPDY_VARIANT(MODE, 512, 1, RMAX), \
+    SPDY_VARIANT(MODE, 128, 4, RMAX), SPDY_VARIANT(MODE, 256, 3, RMAX), SPDY_VARIANT(MODE, 512, 1, RMAX), \
     SPDY_VARIANT(MODE, 1024, 1, 16), SPDY_VARIANT(MODE, 128, 6, 8), SPDY_VARIANT(MODE, 256, 3, 8),       \
     SPDY_VARIANT(MODE, 512, 1, 8), SPDY_VARIANT(MODE, 1024, 1, 8)
 
@@ -1922,6 +1979,56 @@ int spdy_quadratic_errors(const float *coeffs_dev, int64_t N, int32_t L, int32_t
     spdy_quadratic_errors_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(coeffs_dev, errors_dev, total, K);
     SPDY_CUDA_TRY(cudaGetLastError());
     return SPDY_OK;
+}
+
+int spdy_probe_peaks(int device, double *lds_reads_per_s, double *cell_updates_alu_per_s)
+{
+    if (device < 0) return SPDY_ERR_INVALID_ARG;
+    DeviceGuard guard;
+    int rc = guard.enter(device);
+    if (rc != SPDY_OK) return rc;
+    int sms = 0;
+    SPDY_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    const int ctas = sms * 8, threads = 256, iters = 20000;
+    float *out = nullptr;
+    cudaEvent_t ev[2] = {nullptr, nullptr};
+    cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&out), static_cast<size_t>(ctas) * threads * sizeof(float));
+    if (err != cudaSuccess) {
+        g_last_cuda_error = static_cast<int>(err);
+        return err == cudaErrorMemoryAllocation ? SPDY_ERR_NO_MEMORY : SPDY_ERR_CUDA;
+    }
+    auto finish = [&](int code) {
+        if (ev[0]) cudaEventDestroy(ev[0]);
+        if (ev[1]) cudaEventDestroy(ev[1]);
+        cudaFree(out);
+        return code;
+    };
+    if (cudaEventCreate(&ev[0]) != cudaSuccess || cudaEventCreate(&ev[1]) != cudaSuccess) return finish(SPDY_ERR_CUDA);
+    double rates[2] = {0.0, 0.0};
+    for (int which = 0; which < 2; ++which) {
+        float best_ms = 0.0f;
+        for (int rep = 0; rep < 4; ++rep) {  // first repetition warms up
+            cudaEventRecord(ev[0], nullptr);
+            if (which == 0) spdy_probe_lds_kernel<<<ctas, threads>>>(out, iters);
+            else spdy_probe_alu_kernel<<<ctas, threads>>>(out, iters, 0.25f, 0.5f);
+            cudaEventRecord(ev[1], nullptr);
+            err = cudaEventSynchronize(ev[1]);
+            if (err == cudaSuccess) err = cudaGetLastError();
+            if (err != cudaSuccess) {
+                g_last_cuda_error = static_cast<int>(err);
+                return finish(SPDY_ERR_CUDA);
+            }
+            float ms = 0.0f;
+            cudaEventElapsedTime(&ms, ev[0], ev[1]);
+            if (rep > 0 && (best_ms == 0.0f || ms < best_ms)) best_ms = ms;
+        }
+        // 8 reads (resp. 16 cell updates: 8 cells x 2 choices) per thread per iteration
+        const double per_thread = which == 0 ? 8.0 : 16.0;
+        rates[which] = per_thread * iters * static_cast<double>(ctas) * threads / (best_ms * 1e-3);
+    }
+    if (lds_reads_per_s) *lds_reads_per_s = rates[0];
+    if (cell_updates_alu_per_s) *cell_updates_alu_per_s = rates[1];
+    return finish(SPDY_OK);
 }
 
 double spdy_time_target(double t_dense, double speedup, double t_base)

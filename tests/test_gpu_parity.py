@@ -420,3 +420,15 @@ def test_host_buffer_path_uploads_in_chunks():
     fwd_dev, _ = plan.last_timing()
     assert 0.5 * fwd_dev < fwd_host < 3.0 * fwd_dev
     plan.close()
+
+
+def test_peak_probes_are_in_range():
+    """The shared-memory probe must land just under 32 reads per clock per SM, the arithmetic probe
+    well above it (otherwise the roofline's binding unit would be misjudged)."""
+    import torch
+
+    lds, alu = binding.probe_peaks(0)
+    props = torch.cuda.get_device_properties(0)
+    per_clk_sm = lds / (props.multi_processor_count * 1.965e9)
+    assert 20.0 < per_clk_sm <= 33.0
+    assert alu > 1.5 * lds
