@@ -432,3 +432,29 @@ def test_peak_probes_are_in_range():
     per_clk_sm = lds / (props.multi_processor_count * 1.965e9)
     assert 20.0 < per_clk_sm <= 33.0
     assert alu > 1.5 * lds
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_nan_inputs_are_contained(fmt):
+    """NaN errors are outside the value domain: the candidate that holds them may come back flagged
+    (self-check word) or as infeasible, but its neighbours in the batch must be unaffected.  Every
+    table access of the walk back is range-checked, so nothing can go out of bounds."""
+    import torch
+
+    wl = W.make_workload(1, N=12)
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+    bad = wl.errors.copy()
+    bad[5, :, :] = np.nan
+    bad[9, 3, 7] = np.nan
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+    p, c, t = binding.solve_batch(plan, torch.from_numpy(bad).cuda())
+    torch.cuda.synchronize()
+    try:
+        plan.check_status()
+    except binding.SpdyError as e:
+        assert e.status == -6
+    plan.check_status()  # the word was cleared by the read above
+    good = [n for n in range(12) if n not in (5, 9)]
+    assert_same((p.cpu().numpy()[good], c.cpu().numpy()[good], t.cpu().numpy()[good]), tuple(x[good] for x in ref))
+    assert t.cpu().numpy()[5] == -1 and (p.cpu().numpy()[5] == 0xFF).all()
+    plan.close()
