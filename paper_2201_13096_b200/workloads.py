@@ -150,9 +150,9 @@ def _candidate_sensitivities(cfg: int, L: int, N: int, start: int = 0) -> np.nda
 
 CONFIG_NAMES = {
     0: "tiny-L8-K4",
-    1: "resnet50-L53-K42-B10000",
-    2: "bert-base-L72-K42-B10000",
-    3: "bert-large-L144-K64-B65536",
+    1: "resnet50-L53-K42",
+    2: "bert-base-L72-K42",
+    3: "bert-large-L144-K64",
     4: "bert-base-sweep",
 }
 
