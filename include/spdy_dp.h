@@ -56,6 +56,10 @@ typedef enum spdy_status {
  *   per cell and runs about 1.35x faster; the table is 4 bytes per cell.
  *   ARG_U8 keeps Algorithm 1's matrix P (the winning choice index), one byte per cell, at the
  *   price of a compare and two selects per cell update.  Use it when workspace is scarce.
+ *   Equal-time choices can be merged here only for candidates whose errors do not fall with the
+ *   choice index inside any group of equal-time choices (always true for Eq. 4's errors with
+ *   non-negative coefficients); a small kernel tests that per candidate, and the others run with one
+ *   slot per choice.  The workspace then carries one extra 256 bytes per candidate.
  */
 typedef enum spdy_table_format {
     SPDY_TABLE_DEFAULT = 0, /* let the plan choose (currently SPDY_TABLE_ROW_F32) */
@@ -97,8 +101,11 @@ typedef struct spdy_plan_info {
     int64_t issued_updates; /* cell updates the kernel actually issues per candidate (span granularity) */
     int64_t nominal_updates;/* L*K*B per candidate, the unit of the headline metric */
     int64_t distinct_updates; /* like useful_updates after choices of a layer with equal times are merged
-                                 into one shift (row-value table only; equals useful_updates otherwise):
-                                 the cell updates the forward pass has to perform */
+                                 into one shift: the cell updates the forward pass has to perform.  With the
+                                 byte table this is the count for candidates that may be merged (see
+                                 spdy_table_format); issued_updates is given for the same table set */
+    int32_t launches_per_wave; /* kernels one wave of candidates launches (2, or 5 with the byte table's two table sets) */
+    int32_t reserved1;
 } spdy_plan_info;
 
 typedef struct spdy_plan spdy_plan; /* opaque; owns only its own small host and device tables */

@@ -42,7 +42,8 @@ class SpdyPlanInfo(ctypes.Structure):
                 ("smem_bytes", ctypes.c_int64), ("table_bytes_per_candidate", ctypes.c_int64),
                 ("band_cells", ctypes.c_int64), ("useful_updates", ctypes.c_int64),
                 ("issued_updates", ctypes.c_int64), ("nominal_updates", ctypes.c_int64),
-                ("distinct_updates", ctypes.c_int64)]
+                ("distinct_updates", ctypes.c_int64), ("launches_per_wave", ctypes.c_int32),
+                ("reserved1", ctypes.c_int32)]
 
     def as_dict(self) -> dict:
         return {name: int(getattr(self, name)) for name, _ in self._fields_}

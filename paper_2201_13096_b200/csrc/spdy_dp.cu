@@ -99,6 +99,8 @@ struct FwdArgs {
     int32_t row_stride;       // floats per shared-memory row buffer
     int32_t pad;              // +inf guard cells on either side of a row: 32 * the largest cells-per-lane
     float *grows;             // row buffers in global memory (GROWS kernels), else null
+    const uint8_t *cand_flags; // per candidate of the wave, or null: run only candidates whose flag == which
+    int32_t which;
 };
 
 __device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
@@ -379,6 +381,9 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         tap_buf = reinterpret_cast<int2 *>(rows + 2 * static_cast<size_t>(args.row_stride));
     }
 
+    // Two table sets may share a wave (see spdy_monotone_flags_kernel): a CTA whose candidate belongs
+    // to the other set leaves at once, before any barrier.
+    if (args.cand_flags && args.cand_flags[blockIdx.x] != args.which) return;
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
@@ -698,6 +703,10 @@ struct BackArgs {
     int64_t n_first;
     int64_t n_count;
     int32_t L, K;
+    const uint8_t *cand_flags; // as in FwdArgs
+    int32_t which;
+    const uint8_t *slot_ptr;    // byte table of slot indices: translate through these lists (else null)
+    const uint8_t *slot_member;
 };
 
 // Walk back through the byte table (end of Algorithm 1): one thread per candidate.
@@ -705,6 +714,7 @@ __global__ void spdy_backtrack_arg_kernel(const BackArgs args)
 {
     const int64_t n_local = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
     if (n_local >= args.n_count) return;
+    if (args.cand_flags && args.cand_flags[n_local] != args.which) return;
     const int64_t n = args.n_first + n_local;
     const int L = args.L, K = args.K;
     uint8_t *prof = args.profile + n * L;
@@ -720,6 +730,9 @@ __global__ void spdy_backtrack_arg_kernel(const BackArgs args)
         const int t_rel = t - ld.lo;
         int k = 0xFF;
         if (ok && t_rel >= 0 && t_rel < ld.width) k = P[ld.rowoff + t_rel];
+        // A table of slot indices: the slot's winner is its first (lowest) member.
+        if (args.slot_member && k < ld.nslots) k = args.slot_member[l * K + args.slot_ptr[l * (K + 1) + k]];
+        else if (args.slot_member) k = 0xFF;
         if (k >= K) {
             ok = false;
             k = 0xFF;
@@ -800,6 +813,41 @@ __global__ void spdy_backtrack_row_kernel(const BackArgs args)
         }
     }
     if ((!ok || t != 0) && lane == 0) atomicExch(args.status, 1);
+}
+
+// With the byte table the winning choice index is stored, so choices of equal time may be merged into
+// one slot only where the merge cannot change the winner: when, inside every group of equal-time
+// choices, the errors do not fall as the index rises.  Then the group's lowest index attains the
+// group's smallest sum at every cell and wins every tie inside the group, and among groups the
+// lowest first member wins - exactly the choice a scan over all choices in ascending order keeps.
+// This kernel tests that condition per candidate (one warp each): flag 1 = merged tables are exact
+// for it, flag 0 = it needs one slot per choice.  slot_ptr / slot_member are the merged lists.
+__global__ void spdy_monotone_flags_kernel(const float *errors, const float *coeffs, const float *qtab,
+                                           const LayerDesc *layers, const uint8_t *slot_ptr,
+                                           const uint8_t *slot_member, uint8_t *flags, int64_t n_first,
+                                           int64_t n_count, int32_t L, int32_t K)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t n_local = (blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x) >> 5;
+    if (n_local >= n_count) return;
+    const int64_t n = n_first + n_local;
+    bool ok = true;
+    for (int l = 0; l < L; ++l) {
+        const int nslots = layers[l].nslots;
+        const uint8_t *ptr = slot_ptr + static_cast<size_t>(l) * (K + 1);
+        const uint8_t *member = slot_member + static_cast<size_t>(l) * K;
+        for (int u = lane; u < nslots; u += 32) {
+            const int j0 = ptr[u], j1 = ptr[u + 1];
+            float prev = choice_error(errors, coeffs, qtab, n, l, member[j0], L, K);
+            for (int j = j0 + 1; j < j1; ++j) {
+                const float e = choice_error(errors, coeffs, qtab, n, l, member[j], L, K);
+                ok = ok && (prev <= e);  // false for NaN as well
+                prev = e;
+            }
+        }
+    }
+    ok = __all_sync(0xffffffffu, ok);
+    if (lane == 0) flags[n_local] = ok ? 1 : 0;
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -974,6 +1022,12 @@ struct spdy_plan {
     int64_t smem_bytes = 0;
     int32_t row_stride = 0, pad = 0;
     bool global_rows = false;  // row buffers live in the workspace, not in shared memory
+    // Byte table only: `merged` is a second plan over the same rows and passes whose slots are groups
+    // of equal-time choices (ordered by their lowest member); candidates for which that is exact run
+    // on it, the others on this plan (see spdy_monotone_flags_kernel).  `merge_first` marks such a
+    // second plan.
+    bool merge_first = false;
+    spdy_plan *merged = nullptr;
     int64_t pitch = 0;  // table cells per candidate
     int64_t band_cells = 0, useful_updates = 0, distinct_updates = 0, issued_updates = 0;
     int32_t max_width = 0;
@@ -1035,6 +1089,8 @@ int64_t cell_bytes(const spdy_plan *p) { return p->table_format == SPDY_TABLE_RO
 // global memory.  Both are multiples of 256 bytes.
 int64_t table_bytes_one(const spdy_plan *p) { return std::max<int64_t>(256, round_up(p->pitch * cell_bytes(p), 256)); }
 int64_t row_bytes_one(const spdy_plan *p) { return p->global_rows ? round_up(2LL * p->row_stride * 4, 256) : 0; }
+// One flag byte per candidate when two table sets share the batch (kept 256-byte granular).
+int64_t flag_bytes_one(const spdy_plan *p) { return p->merged ? 256 : 0; }
 
 // Live band of every row and the range of every (layer, choice) pair.
 //   lo_l = sum_{j<=l} mn_j,  hi_l = min(B, sum_{j<=l} mx_j, B - sum_{j>l} mn_j)
@@ -1098,7 +1154,9 @@ int build_bands(spdy_plan *p)
 
 // Shift slots of every layer (see TapRange).  With `merge` the usable choices of a layer are
 // grouped by time, slots in ascending time order; without it slot u is choice u.
-void build_slots(spdy_plan *p, bool merge)
+// merge: 0 = slot u is choice u; 1 = groups of equal time in ascending time order (row-value
+// table); 2 = groups of equal time in the order of their lowest member (byte table, second plan).
+void build_slots(spdy_plan *p, int merge)
 {
     const int L = p->L, K = p->K;
     p->slots.assign(static_cast<size_t>(L) * K, TapRange{0, -1});
@@ -1125,6 +1183,22 @@ void build_slots(spdy_plan *p, bool merge)
                 if (taps[k].b >= taps[k].a) order[usable++] = k;
             std::stable_sort(order.begin(), order.begin() + usable,
                              [&](int x, int y) { return taps[x].a < taps[y].a; });
+            if (merge == 2) {
+                // groups (runs of equal shift in `order`, members ascending) re-ordered by first member
+                std::vector<std::pair<int, int>> runs;  // [begin, end) in `order`
+                for (int i = 0; i < usable;) {
+                    int j = i + 1;
+                    while (j < usable && taps[order[j]].a == taps[order[i]].a) ++j;
+                    runs.emplace_back(i, j);
+                    i = j;
+                }
+                std::sort(runs.begin(), runs.end(),
+                          [&](const std::pair<int, int> &x, const std::pair<int, int> &y) { return order[x.first] < order[y.first]; });
+                std::vector<int> reordered;
+                for (const auto &r : runs)
+                    for (int i = r.first; i < r.second; ++i) reordered.push_back(order[i]);
+                std::copy(reordered.begin(), reordered.end(), order.begin());
+            }
             for (int i = 0; i < usable; ++i) {
                 const int k = order[i];
                 if (nslots == 0 || slots[nslots - 1].a != taps[k].a) {
@@ -1373,7 +1447,7 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
         if (!(row_mode || arg_mode)) return SPDY_ERR_INVALID_ARG;
         if (row_mode != (p->table_format == SPDY_TABLE_ROW_F32)) return SPDY_ERR_INVALID_ARG;
     }
-    build_slots(p, p->mode == MODE_ROW || p->mode == MODE_ROW2);
+    build_slots(p, (p->mode == MODE_ROW || p->mode == MODE_ROW2) ? 1 : (p->merge_first ? 2 : 0));
     p->cluster = 1;
     if (opts && opts->cluster != 0 && opts->cluster != 1 && opts->cluster != 2 && opts->cluster != 4 &&
         opts->cluster != 8)
@@ -1556,8 +1630,12 @@ const char *spdy_strerror(int status)
     }
 }
 
-int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int32_t K, int32_t B,
-                     int device, const spdy_options *opts)
+}  // extern "C"
+
+namespace {
+
+int create_plan(spdy_plan **out, const int32_t *times_host, int32_t L, int32_t K, int32_t B, int device,
+                const spdy_options *opts, bool merge_first)
 {
     if (!out) return SPDY_ERR_INVALID_ARG;
     *out = nullptr;
@@ -1574,6 +1652,7 @@ int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int3
     p->K = K;
     p->B = B;
     p->device = device;
+    p->merge_first = merge_first;
     int rc = SPDY_OK;
     try {
         p->times.assign(times_host, times_host + static_cast<size_t>(L) * K);
@@ -1594,9 +1673,43 @@ int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int3
     return SPDY_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int32_t K, int32_t B,
+                     int device, const spdy_options *opts)
+{
+    int rc = create_plan(out, times_host, L, K, B, device, opts, false);
+    if (rc != SPDY_OK) return rc;
+    spdy_plan *p = *out;
+    // Byte table, one CTA per candidate: add the second plan with merged equal-time choices when
+    // merging removes any work.  It must lay out rows, passes and table exactly like the first.
+    if (p->table_format == SPDY_TABLE_ARG_U8 && p->cluster == 1 && p->feasible) {
+        spdy_options o = {};
+        if (opts) o = *opts;
+        o.table_format = SPDY_TABLE_ARG_U8;
+        o.threads = p->threads;
+        o.cluster = 1;
+        o.forward_mode = p->mode;
+        o.rows_in_global = p->global_rows ? 1 : 0;
+        spdy_plan *m = nullptr;
+        if (create_plan(&m, times_host, L, K, B, device, &o, true) == SPDY_OK) {
+            const bool same_shape = m->pitch == p->pitch && m->row_stride == p->row_stride && m->pad == p->pad &&
+                                    m->threads == p->threads && m->smem_bytes == p->smem_bytes &&
+                                    m->global_rows == p->global_rows && m->variant == p->variant;
+            if (same_shape && m->distinct_updates < p->distinct_updates) p->merged = m;
+            else spdy_plan_destroy(m);
+        }
+    }
+    return SPDY_OK;
+}
+
 void spdy_plan_destroy(spdy_plan *plan)
 {
     if (!plan) return;
+    if (plan->merged) spdy_plan_destroy(plan->merged);
+    plan->merged = nullptr;
     if (plan->d_blob || plan->d_arena) {
         DeviceGuard guard;
         guard.enter(plan->device);
@@ -1631,7 +1744,9 @@ int spdy_plan_get_info(const spdy_plan *plan, spdy_plan_info *info)
     info->band_cells = plan->band_cells;
     info->useful_updates = plan->useful_updates;
     info->issued_updates = plan->issued_updates;
-    info->distinct_updates = plan->distinct_updates;
+    info->distinct_updates = plan->merged ? plan->merged->distinct_updates : plan->distinct_updates;
+    if (plan->merged) info->issued_updates = plan->merged->issued_updates;
+    info->launches_per_wave = plan->merged ? 5 : 2;
     info->nominal_updates = static_cast<int64_t>(plan->L) * plan->K * plan->B;
     return SPDY_OK;
 }
@@ -1649,7 +1764,7 @@ int spdy_plan_get_bands(const spdy_plan *plan, int32_t *lo_host, int32_t *width_
 size_t spdy_workspace_bytes(const spdy_plan *plan, int64_t N)
 {
     if (!plan || N <= 0) return 0;
-    return static_cast<size_t>(table_bytes_one(plan) + row_bytes_one(plan)) * static_cast<size_t>(N);
+    return static_cast<size_t>(table_bytes_one(plan) + row_bytes_one(plan) + flag_bytes_one(plan)) * static_cast<size_t>(N);
 }
 
 }  // extern "C"
@@ -1703,77 +1818,108 @@ int solve_impl(const spdy_plan *plan, const float *errors_dev, const float *coef
             mplan->events_used += 3;
             SPDY_CUDA_TRY(cudaEventRecord(ev[0], stream));
         }
-        FwdArgs fa;
-        fa.errors = errors_dev;
-        fa.coeffs = coeffs_dev;
-        fa.qtab = plan->d_qtab;
-        fa.slots = plan->d_slots;
-        fa.slot_ptr = plan->d_slot_ptr;
-        fa.slot_member = plan->d_slot_member;
-        fa.layers = plan->d_layers;
-        fa.span_masks = plan->d_masks;
-        fa.span_kranges = plan->d_kranges;
-        fa.table = workspace_dev;
-        fa.cost = cost_dev;
-        fa.time_used = time_used_dev;
-        fa.pitch = pitch_cells;
-        fa.n_first = first;
-        fa.L = plan->L;
-        fa.K = plan->K;
-        fa.row_stride = plan->row_stride;
-        fa.pad = plan->pad;
-        fa.grows = grows;
-        // Grid x is limited to 2^31-1 CTAs, far above any wave that fits in memory.
-        if (plan->cluster > 1) {
-            ClusterArgs ca;
-            ca.f = fa;
-            ca.slices = plan->d_slices;
-            ca.C = plan->cluster;
-            ca.out_stride = plan->out_stride;
-            ca.win_stride = plan->win_stride;
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(static_cast<unsigned>(count * plan->cluster), 1, 1);
-            cfg.blockDim = dim3(static_cast<unsigned>(plan->threads), 1, 1);
-            cfg.dynamicSmemBytes = static_cast<size_t>(plan->smem_bytes);
-            cfg.stream = stream;
-            cudaLaunchAttribute attr;
-            attr.id = cudaLaunchAttributeClusterDimension;
-            attr.val.clusterDim.x = static_cast<unsigned>(plan->cluster);
-            attr.val.clusterDim.y = 1;
-            attr.val.clusterDim.z = 1;
-            cfg.attrs = &attr;
-            cfg.numAttrs = 1;
-            SPDY_CUDA_TRY(cudaLaunchKernelEx(&cfg, plan->cvariant->fn, ca));
-        } else {
-            plan->variant->fn<<<static_cast<unsigned>(count), plan->threads, static_cast<size_t>(plan->smem_bytes), stream>>>(fa);
+        // With a second (merged) table set every candidate of the wave gets a flag saying which set is
+        // exact for it; both sets are then launched over the whole wave and every CTA / walk-back thread
+        // runs only if its candidate carries the set's flag (the others leave at once).
+        uint8_t *flags = nullptr;
+        if (plan->merged) {
+            flags = static_cast<unsigned char *>(workspace_dev) + wave * (table_bytes_one(plan) + row_bytes_one(plan));
+            const spdy_plan *m = plan->merged;
+            const int bt = 128;
+            spdy_monotone_flags_kernel<<<static_cast<unsigned>((count * 32 + bt - 1) / bt), bt, 0, stream>>>(
+                errors_dev, coeffs_dev, m->d_qtab, m->d_layers, m->d_slot_ptr, m->d_slot_member, flags, first, count,
+                plan->L, plan->K);
+            SPDY_CUDA_TRY(cudaGetLastError());
         }
-        SPDY_CUDA_TRY(cudaGetLastError());
+        auto forward = [&](const spdy_plan *tp, int which) -> int {
+            FwdArgs fa;
+            fa.errors = errors_dev;
+            fa.coeffs = coeffs_dev;
+            fa.qtab = tp->d_qtab;
+            fa.slots = tp->d_slots;
+            fa.slot_ptr = tp->d_slot_ptr;
+            fa.slot_member = tp->d_slot_member;
+            fa.layers = tp->d_layers;
+            fa.span_masks = tp->d_masks;
+            fa.span_kranges = tp->d_kranges;
+            fa.table = workspace_dev;
+            fa.cost = cost_dev;
+            fa.time_used = time_used_dev;
+            fa.pitch = pitch_cells;
+            fa.n_first = first;
+            fa.L = tp->L;
+            fa.K = tp->K;
+            fa.row_stride = tp->row_stride;
+            fa.pad = tp->pad;
+            fa.grows = grows;
+            fa.cand_flags = flags;
+            fa.which = which;
+            // Grid x is limited to 2^31-1 CTAs, far above any wave that fits in memory.
+            if (tp->cluster > 1) {
+                ClusterArgs ca;
+                ca.f = fa;
+                ca.slices = tp->d_slices;
+                ca.C = tp->cluster;
+                ca.out_stride = tp->out_stride;
+                ca.win_stride = tp->win_stride;
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(static_cast<unsigned>(count * tp->cluster), 1, 1);
+                cfg.blockDim = dim3(static_cast<unsigned>(tp->threads), 1, 1);
+                cfg.dynamicSmemBytes = static_cast<size_t>(tp->smem_bytes);
+                cfg.stream = stream;
+                cudaLaunchAttribute attr;
+                attr.id = cudaLaunchAttributeClusterDimension;
+                attr.val.clusterDim.x = static_cast<unsigned>(tp->cluster);
+                attr.val.clusterDim.y = 1;
+                attr.val.clusterDim.z = 1;
+                cfg.attrs = &attr;
+                cfg.numAttrs = 1;
+                SPDY_CUDA_TRY(cudaLaunchKernelEx(&cfg, tp->cvariant->fn, ca));
+            } else {
+                tp->variant->fn<<<static_cast<unsigned>(count), tp->threads, static_cast<size_t>(tp->smem_bytes), stream>>>(fa);
+            }
+            SPDY_CUDA_TRY(cudaGetLastError());
+            return SPDY_OK;
+        };
+        auto walk_back = [&](const spdy_plan *tp, int which) -> int {
+            BackArgs ba;
+            ba.errors = errors_dev;
+            ba.coeffs = coeffs_dev;
+            ba.qtab = tp->d_qtab;
+            ba.times = tp->d_times;
+            ba.layers = tp->d_layers;
+            ba.table = workspace_dev;
+            ba.cost = cost_dev;
+            ba.time_used = time_used_dev;
+            ba.profile = profile_dev;
+            ba.status = plan->d_status;  // one self-check word per public plan
+            ba.pitch = pitch_cells;
+            ba.n_first = first;
+            ba.n_count = count;
+            ba.L = tp->L;
+            ba.K = tp->K;
+            ba.cand_flags = flags;
+            ba.which = which;
+            ba.slot_ptr = tp->merge_first ? tp->d_slot_ptr : nullptr;
+            ba.slot_member = tp->merge_first ? tp->d_slot_member : nullptr;
+            if (tp->table_format == SPDY_TABLE_ARG_U8) {
+                const int bt = 64;
+                spdy_backtrack_arg_kernel<<<static_cast<unsigned>((count + bt - 1) / bt), bt, 0, stream>>>(ba);
+            } else {
+                const int bt = 128;  // 4 warps = 4 candidates per CTA
+                spdy_backtrack_row_kernel<<<static_cast<unsigned>((count * 32 + bt - 1) / bt), bt, 0, stream>>>(ba);
+            }
+            SPDY_CUDA_TRY(cudaGetLastError());
+            return SPDY_OK;
+        };
+        int lrc = SPDY_OK;
+        if (plan->merged) lrc = forward(plan->merged, 1);
+        if (lrc == SPDY_OK) lrc = forward(plan, 0);
+        if (lrc != SPDY_OK) return lrc;
         if (ev) SPDY_CUDA_TRY(cudaEventRecord(ev[1], stream));
-
-        BackArgs ba;
-        ba.errors = errors_dev;
-        ba.coeffs = coeffs_dev;
-        ba.qtab = plan->d_qtab;
-        ba.times = plan->d_times;
-        ba.layers = plan->d_layers;
-        ba.table = workspace_dev;
-        ba.cost = cost_dev;
-        ba.time_used = time_used_dev;
-        ba.profile = profile_dev;
-        ba.status = plan->d_status;
-        ba.pitch = pitch_cells;
-        ba.n_first = first;
-        ba.n_count = count;
-        ba.L = plan->L;
-        ba.K = plan->K;
-        if (plan->table_format == SPDY_TABLE_ARG_U8) {
-            const int bt = 64;
-            spdy_backtrack_arg_kernel<<<static_cast<unsigned>((count + bt - 1) / bt), bt, 0, stream>>>(ba);
-        } else {
-            const int bt = 128;  // 4 warps = 4 candidates per CTA
-            spdy_backtrack_row_kernel<<<static_cast<unsigned>((count * 32 + bt - 1) / bt), bt, 0, stream>>>(ba);
-        }
-        SPDY_CUDA_TRY(cudaGetLastError());
+        if (plan->merged) lrc = walk_back(plan->merged, 1);
+        if (lrc == SPDY_OK) lrc = walk_back(plan, 0);
+        if (lrc != SPDY_OK) return lrc;
         if (ev) SPDY_CUDA_TRY(cudaEventRecord(ev[2], stream));
     }
     return SPDY_OK;

@@ -458,3 +458,40 @@ def test_nan_inputs_are_contained(fmt):
     assert_same((p.cpu().numpy()[good], c.cpu().numpy()[good], t.cpu().numpy()[good]), tuple(x[good] for x in ref))
     assert t.cpu().numpy()[5] == -1 and (p.cpu().numpy()[5] == 0xFF).all()
     plan.close()
+
+
+def test_byte_table_merges_equal_time_choices_only_where_exact():
+    """With the uint8 table, candidates whose errors rise with the choice index inside every group of
+    equal-time choices run on merged slots, the others on one slot per choice - in one batch."""
+    import torch
+
+    wl = W.make_workload(4, N=40, B=1000)  # many equal times after rounding
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=binding.SPDY_TABLE_ARG_U8)
+    info = plan.info
+    assert info["launches_per_wave"] == 5 and info["distinct_updates"] < info["useful_updates"]
+    errors = wl.errors.copy()
+    rng = np.random.default_rng(12)
+    for n in range(0, 40, 3):  # every third candidate: errors in random order, some equal
+        errors[n] = rng.permuted(errors[n], axis=1)
+        errors[n, :, 5] = errors[n, :, 6]
+    for n in range(1, 40, 7):  # flat errors: every choice ties
+        errors[n] = np.float32(0.5)
+    ref = oracle.solve_batch(errors, wl.times, wl.B, threads=CORES)
+    p, c, t = binding.solve_batch(plan, torch.from_numpy(errors).cuda())
+    torch.cuda.synchronize()
+    plan.check_status()
+    assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), ref)
+    ws = torch.empty(plan.workspace_bytes(7), dtype=torch.uint8, device="cuda")  # several waves
+    p, c, t = binding.solve_batch(plan, torch.from_numpy(errors).cuda(), workspace=ws)
+    torch.cuda.synchronize()
+    assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), ref)
+    plan.close()
+    # coefficients of either sign: negative ones make Eq. 4's errors fall with the index
+    coeffs = rng.normal(size=(30, wl.L)).astype(np.float32)
+    ref = oracle.solve_batch(oracle.quadratic_errors(coeffs, wl.K), wl.times, wl.B, threads=CORES)
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=binding.SPDY_TABLE_ARG_U8)
+    p, c, t = binding.solve_batch_coeffs(plan, torch.from_numpy(coeffs).cuda())
+    torch.cuda.synchronize()
+    plan.check_status()
+    assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), ref)
+    plan.close()

@@ -91,9 +91,12 @@ def test_bands_of_the_named_configs(cfg):
     assert info["nominal_updates"] == wl.L * wl.K * wl.B
     assert 0 < info["distinct_updates"] <= info["useful_updates"] <= info["nominal_updates"] + wl.L * wl.K
     assert info["distinct_updates"] <= info["issued_updates"]
-    # the byte table keeps one slot per choice: nothing is merged
+    # the byte table merges the same groups (for candidates where that is exact) in a second table set
     arg = binding.Plan(wl.times, wl.B, device=-1, table_format=binding.SPDY_TABLE_ARG_U8).info
-    assert arg["distinct_updates"] == arg["useful_updates"] == info["useful_updates"] <= arg["issued_updates"]
+    assert arg["useful_updates"] == info["useful_updates"]
+    assert arg["distinct_updates"] == info["distinct_updates"] <= arg["issued_updates"]
+    assert arg["launches_per_wave"] == (5 if arg["distinct_updates"] < arg["useful_updates"] else 2)
+    assert info["launches_per_wave"] == 2
     # merged work recomputed from the timing table: one shift per distinct usable time of a layer
     lo_prev, w_prev, distinct = 0, 1, 0
     for l in range(wl.L):
