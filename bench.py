@@ -31,8 +31,8 @@ CELLS_PER_CLK_PER_SM = 32.0  # one 4-byte shared-memory read per cell update, 32
 # DRAM bytes (read + write) of the forward kernel per candidate from an ncu capture of one wave
 # (592 candidates) of the BERT-base shape; traffic grows in proportion to N.  Valid only for the
 # library version the counters were taken with.
-NCU_TRAFFIC = {"version": 1003, "workload_prefix": "bert-base-L72-K42",
-               "bytes_per_candidate": {"row_f32": 762.88e6 / 592, "arg_u8": 153.30e6 / 592}}
+NCU_TRAFFIC = {"version": 1004, "workload_prefix": "bert-base-L72-K42",
+               "bytes_per_candidate": {"row_f32": 762.88e6 / 592, "arg_u8": 154.26e6 / 592}}
 
 
 def parse_args():

@@ -1611,7 +1611,7 @@ struct DeviceGuard {
 
 extern "C" {
 
-int spdy_version(void) { return 1003; }
+int spdy_version(void) { return 1004; }
 
 int spdy_last_cuda_error(void) { return g_last_cuda_error; }
 
