@@ -52,6 +52,10 @@ def parse_args():
     ap.add_argument("--search", type=int, default=0, metavar="TRIALS",
                     help="also run Algorithm 4 with this many trials per loop on the workload's timing table "
                          "(synthetic loss) and report where the time goes, under the key 'search'")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of one line: every named shape and sweep point (N in 1..65536, B in 10^3..10^5), "
+                         "each with its oracle sample and a bit-exact check; prints one JSON line per point and a "
+                         "markdown table on stderr")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="CPU work budget of the oracle legs")
@@ -404,9 +408,102 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+SWEEP_POINTS = [  # (config, N, B override)
+    (4, 1, None), (4, 16, None), (4, 256, None), (4, 4096, None), (4, 65536, None),
+    (4, 4096, 1000), (4, 4096, 100000), (1, None, None), (2, None, None), (3, None, None),
+]
+
+
+def run_sweep(args):
+    """Every named shape and sweep point on one GPU: device-resident timing, the oracle on a bounded
+    sample of the same candidates (timed, and compared bit for bit with the GPU's outputs)."""
+    import torch
+
+    import oracle
+    from paper_2201_13096_b200 import binding, workloads as W
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the solver has no CPU path")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    cores = host_cores()
+    lds_peak, _ = binding.probe_peaks(0)
+    fmt = {"default": 0, "arg": 1, "row": 2}[args.table]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    rows = []
+    for cfg, n, budget in SWEEP_POINTS:
+        wl = W.make_workload(cfg, N=n, B=budget)
+        plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+        info = plan.info
+        plan.enable_timing(True)
+        errors = torch.from_numpy(wl.errors).to(dev)
+        ws = torch.empty(max(256, min(plan.workspace_bytes(wl.N), 48 << 30)), dtype=torch.uint8, device=dev)
+        out = None
+        fwd, back, total = [], [], []
+        for it in range(3 + 5):
+            flush.fill_(it)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            out = binding.solve_batch(plan, errors, workspace=ws)
+            b.record()
+            f, w = plan.last_timing()
+            if it >= 3:
+                fwd.append(f)
+                back.append(w)
+                total.append(a.elapsed_time(b))
+        plan.check_status()
+        ms, f_ms = float(np.mean(total)), float(np.mean(fwd))
+        # oracle: single-core time of one candidate, then a bounded sample on all cores, compared
+        t0 = time.perf_counter()
+        oracle.solve_batch(wl.errors[:1], wl.times, wl.B, threads=1)
+        one = time.perf_counter() - t0
+        k = int(min(wl.N, max(cores, 1.5 * cores / max(one, 1e-6))))  # about 1.5 s of oracle work per point
+        sample = np.sort(np.random.default_rng(1).choice(wl.N, size=k, replace=False))
+        t0 = time.perf_counter()
+        ref = oracle.solve_batch(wl.errors[sample], wl.times, wl.B, threads=min(cores, k))
+        dt = time.perf_counter() - t0
+        p, c, t = (x.cpu().numpy() for x in out)
+        exact = bool(np.array_equal(p[sample], ref[0]) and c[sample].tobytes() == ref[1].tobytes()
+                     and np.array_equal(t[sample], ref[2]))
+        cellb = 4 if info["table_format"] == 2 else 1
+        hbm_bytes = wl.N * (info["band_cells"] * cellb + wl.L * wl.K * 4)
+        row = {"workload": wl.name, "N": wl.N, "L": wl.L, "K": wl.K, "B": wl.B,
+               "table_format": {1: "arg_u8", 2: "row_f32"}[info["table_format"]],
+               "threads": info["threads"], "cluster": info["cluster"], "rows_in_global": info["rows_in_global"],
+               "gpu_ms": ms, "forward_ms": f_ms, "walkback_ms": float(np.mean(back)),
+               "candidates_per_s": wl.N / (ms * 1e-3),
+               "nominal_cell_updates_per_s": wl.N * info["nominal_updates"] / (ms * 1e-3),
+               "executed_cell_updates_per_s": wl.N * info["distinct_updates"] / (f_ms * 1e-3),
+               "roofline_frac_of_measured_lds": wl.N * info["distinct_updates"] / (f_ms * 1e-3) / lds_peak,
+               "table_and_errors_gb_per_s": hbm_bytes / (f_ms * 1e-3) / 1e9,
+               "oracle_ms_per_candidate_one_core": 1e3 * one,
+               "oracle_candidates_per_s_all_cores": k / dt, "oracle_cores": min(cores, k), "oracle_sample": k,
+               "bit_exact_on_sample": exact}
+        rows.append(row)
+        print(json.dumps(row), flush=True)
+        plan.close()
+        del errors, ws
+        torch.cuda.empty_cache()
+    head = ("| workload | table | CTA | GPU ms | candidates/s | nominal upd/s | executed upd/s | frac | table+errors GB/s "
+            "| oracle ms (1 core) | oracle cand/s (cores) | bit-exact (sample) |")
+    print(head, file=sys.stderr)
+    print("|" + "---|" * 12, file=sys.stderr)
+    for r in rows:
+        shape = f'{r["threads"]} thr' + (f' x{r["cluster"]}' if r["cluster"] > 1 else "") + (", rows in global" if r["rows_in_global"] else "")
+        print(f'| {r["workload"]} | {r["table_format"]} | {shape} | {r["gpu_ms"]:.3f} | {r["candidates_per_s"]:.4g} | '
+              f'{r["nominal_cell_updates_per_s"]:.3g} | {r["executed_cell_updates_per_s"]:.3g} | '
+              f'{r["roofline_frac_of_measured_lds"]:.3f} | {r["table_and_errors_gb_per_s"]:.0f} | '
+              f'{r["oracle_ms_per_candidate_one_core"]:.2f} | {r["oracle_candidates_per_s_all_cores"]:.4g} ({r["oracle_cores"]}) | '
+              f'{"yes" if r["bit_exact_on_sample"] else "NO"} ({r["oracle_sample"]}) |', file=sys.stderr)
+    if not all(r["bit_exact_on_sample"] for r in rows):
+        raise SystemExit("a sweep point disagrees with the oracle")
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
