@@ -167,3 +167,20 @@ def test_wide_rows_leave_shared_memory():
     for c in (2, 4, 8):
         info = binding.Plan(small.times, small.B, device=-1, cluster=c).info
         assert info["cluster"] == c and info["distinct_updates"] <= info["issued_updates"]
+
+
+def test_option_validation_of_the_newer_fields():
+    t = np.ones((3, 4), np.int32)
+    with pytest.raises(binding.SpdyError):
+        binding.Plan(t, 10, device=-1, rows_in_global=2)
+    with pytest.raises(binding.SpdyError):
+        binding.Plan(t, 10, device=-1, rows_in_global=1, cluster=2)
+    info = binding.Plan(t, 10, device=-1, rows_in_global=1).info
+    assert info["rows_in_global"] == 1 and info["threads"] == 1024 and info["table_bytes_per_candidate"] % 256 == 0
+    # equal times everywhere: the byte table gets its merged table set, the row table merges always
+    arg = binding.Plan(t, 10, device=-1, table_format=binding.SPDY_TABLE_ARG_U8).info
+    row = binding.Plan(t, 10, device=-1).info
+    assert arg["launches_per_wave"] == 5 and row["launches_per_wave"] == 2
+    assert arg["distinct_updates"] == row["distinct_updates"] < row["useful_updates"]
+    distinct = np.arange(12, dtype=np.int32).reshape(3, 4)  # no two choices of a layer share a time
+    assert binding.Plan(distinct, 20, device=-1, table_format=binding.SPDY_TABLE_ARG_U8).info["launches_per_wave"] == 2
