@@ -53,7 +53,8 @@ typedef enum spdy_status {
  *   ROW_F32 keeps Algorithm 1's matrix D (the row values) and lets the walk back re-derive, at
  *   each of the L cells it visits, the lowest k whose fp32 sum D_{l-1}[t - times[l][k]] +
  *   errors[n][l][k] equals D_l[t] bit for bit.  The forward pass then needs only add + minimum
- *   per cell and runs about 1.35x faster; the table is 4 bytes per cell.
+ *   per cell, merges choices of equal time unconditionally, and runs about 1.3x faster; the table is
+ *   4 bytes per cell.
  *   ARG_U8 keeps Algorithm 1's matrix P (the winning choice index), one byte per cell, at the
  *   price of a compare and two selects per cell update.  Use it when workspace is scarce.
  *   Equal-time choices can be merged here only for candidates whose errors do not fall with the
@@ -70,15 +71,18 @@ typedef enum spdy_table_format {
 typedef struct spdy_options {
     int32_t table_format;  /* spdy_table_format */
     int32_t threads;       /* threads per CTA, 0 = choose; one of 128, 256, 512, 1024 and >= K */
-    int32_t cluster;       /* CTAs cooperating on one candidate, 0 = choose; 1, 2, 4 or 8 */
+    int32_t cluster;       /* CTAs cooperating on one candidate: 0 or 1 = one CTA (the default); 2, 4 or 8 = a
+                              thread-block cluster that splits every row, which shortens the latency of
+                              batches with fewer candidates than SMs.  1 also forbids the fallbacks for
+                              rows too wide for one CTA's shared memory (UNSUPPORTED instead) */
     int32_t forward_mode;  /* 0 = choose.  Variants of the forward kernel's cell update, all with
                               identical results, for measurement: 1 compare+select (ARG_U8),
                               2 compare+predicated moves (ARG_U8), 3 fp32 minimum (ROW_F32),
                               4 packed adds + 3-input minimum over choice pairs (ROW_F32) */
     int32_t rows_in_global; /* 1: keep the two dynamic-program rows in the workspace (global memory) rather than
-                              in shared memory.  Chosen automatically when a band is too wide even for a
-                              cluster of 8 CTAs (B beyond a few 10^5 buckets); slower, but any width runs.
-                              One CTA of 1024 threads per candidate; not combinable with cluster > 1 */
+                              in shared memory and read them through L1.  Chosen automatically when two rows
+                              do not fit one CTA's shared memory (B of about 10^5 buckets and more); any width
+                              runs.  One CTA of 1024 threads per candidate; not combinable with cluster > 1 */
     int32_t reserved[3];   /* must be 0 */
 } spdy_options;
 
@@ -120,7 +124,7 @@ typedef struct spdy_plan spdy_plan; /* opaque; owns only its own small host and 
  *   opts        host, may be NULL for defaults.
  *   *out        receives the plan; destroy with spdy_plan_destroy.
  * Errors: INVALID_ARG (null, L<1, K<1, K>255, B<0, a negative time, bad option), UNSUPPORTED
- * (band too wide for the device's shared memory at the largest cluster), NO_MEMORY, CUDA.
+ * (band too wide for the launch shape the options pin), NO_MEMORY, CUDA.
  */
 int spdy_plan_create(spdy_plan **out, const int32_t *times_host, int32_t L, int32_t K, int32_t B,
                      int device, const spdy_options *opts);
