@@ -1772,9 +1772,11 @@ size_t spdy_workspace_bytes(const spdy_plan *plan, int64_t N)
 namespace {
 
 // The whole path for one batch; exactly one of errors_dev / coeffs_dev is non-null.
+// phases: bit 0 = forward pass (and final minimum), bit 1 = walk back; the host-buffer path runs them
+// separately so that one walk back serves several forward launches into one table.
 int solve_impl(const spdy_plan *plan, const float *errors_dev, const float *coeffs_dev, int64_t N,
                uint8_t *profile_dev, float *cost_dev, int32_t *time_used_dev, void *workspace_dev,
-               size_t workspace_bytes, void *cuda_stream, bool keep_timing = false)
+               size_t workspace_bytes, void *cuda_stream, bool keep_timing = false, int phases = 3)
 {
     if (!plan || plan->device < 0 || N < 0) return SPDY_ERR_INVALID_ARG;
     if (N == 0) return SPDY_OK;
@@ -1822,8 +1824,8 @@ int solve_impl(const spdy_plan *plan, const float *errors_dev, const float *coef
         // exact for it; both sets are then launched over the whole wave and every CTA / walk-back thread
         // runs only if its candidate carries the set's flag (the others leave at once).
         uint8_t *flags = nullptr;
-        if (plan->merged) {
-            flags = static_cast<unsigned char *>(workspace_dev) + wave * (table_bytes_one(plan) + row_bytes_one(plan));
+        if (plan->merged) flags = static_cast<unsigned char *>(workspace_dev) + wave * (table_bytes_one(plan) + row_bytes_one(plan));
+        if (plan->merged && (phases & 1)) {
             const spdy_plan *m = plan->merged;
             const int bt = 128;
             spdy_monotone_flags_kernel<<<static_cast<unsigned>((count * 32 + bt - 1) / bt), bt, 0, stream>>>(
@@ -1913,13 +1915,17 @@ int solve_impl(const spdy_plan *plan, const float *errors_dev, const float *coef
             return SPDY_OK;
         };
         int lrc = SPDY_OK;
-        if (plan->merged) lrc = forward(plan->merged, 1);
-        if (lrc == SPDY_OK) lrc = forward(plan, 0);
-        if (lrc != SPDY_OK) return lrc;
+        if (phases & 1) {
+            if (plan->merged) lrc = forward(plan->merged, 1);
+            if (lrc == SPDY_OK) lrc = forward(plan, 0);
+            if (lrc != SPDY_OK) return lrc;
+        }
         if (ev) SPDY_CUDA_TRY(cudaEventRecord(ev[1], stream));
-        if (plan->merged) lrc = walk_back(plan->merged, 1);
-        if (lrc == SPDY_OK) lrc = walk_back(plan, 0);
-        if (lrc != SPDY_OK) return lrc;
+        if (phases & 2) {
+            if (plan->merged) lrc = walk_back(plan->merged, 1);
+            if (lrc == SPDY_OK) lrc = walk_back(plan, 0);
+            if (lrc != SPDY_OK) return lrc;
+        }
         if (ev) SPDY_CUDA_TRY(cudaEventRecord(ev[2], stream));
     }
     return SPDY_OK;
@@ -2044,8 +2050,9 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
     // An error table goes up in chunks of growing size (one full wave of CTAs first, then six times
     // the previous chunk) on a second stream, so that every upload but the first hides behind the
     // kernels of the chunk before it; an upload takes about a seventh of the time its candidates take
-    // to solve.  Every chunk costs one more latency-bound walk-back launch, so chunks are few, and
-    // coefficient input (K times smaller) goes up in one piece.
+    // to solve.  Every chunk boundary costs a launch tail (and a walk back, unless one serves all), so
+    // chunks are few - one wave, then the rest, measured best at the BERT-base shape - and coefficient
+    // input (K times smaller) goes up in one piece.
     const int64_t per_cand = static_cast<int64_t>(plan->L) * (coeffs ? 1 : plan->K);
     std::vector<int64_t> bounds(1, 0);
     {
@@ -2078,16 +2085,31 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
     } else {
         SPDY_CUDA_TRY(cudaMemcpyAsync(d_err, errors_host, err_bytes, cudaMemcpyHostToDevice, stream));
     }
+    // When the whole batch's table fits the staging workspace (and nothing but tables lives there),
+    // the chunks' forward passes write disjoint parts of it and ONE walk back follows: the walk back
+    // is a latency chain of L steps whatever the number of candidates.
+    const bool one_walk_back = chunks > 1 && plan->feasible && !plan->merged && !plan->global_rows &&
+                               ws_bytes >= ws_one * static_cast<size_t>(N);
     for (size_t c = 0; c < chunks; ++c) {
         const int64_t first = bounds[c], count = bounds[c + 1] - bounds[c];
         if (chunks > 1) SPDY_CUDA_TRY(cudaStreamWaitEvent(stream, plan->copy_events[c], 0));
         const float *in = d_err + first * per_cand;
-        rc = solve_impl(plan, coeffs ? nullptr : in, coeffs ? in : nullptr, count, d_profile + first * plan->L,
-                        d_cost + first, d_time + first, base + off_ws, ws_bytes, stream, c > 0);
+        if (one_walk_back)
+            rc = solve_impl(plan, coeffs ? nullptr : in, coeffs ? in : nullptr, count, d_profile + first * plan->L,
+                            d_cost + first, d_time + first, base + off_ws + static_cast<size_t>(first) * ws_one,
+                            static_cast<size_t>(count) * ws_one, stream, c > 0, 1);
+        else
+            rc = solve_impl(plan, coeffs ? nullptr : in, coeffs ? in : nullptr, count, d_profile + first * plan->L,
+                            d_cost + first, d_time + first, base + off_ws, ws_bytes, stream, c > 0);
         if (rc != SPDY_OK) {
             if (chunks > 1) cudaStreamSynchronize(plan->copy_stream);
             return rc;
         }
+    }
+    if (one_walk_back) {
+        rc = solve_impl(plan, coeffs ? nullptr : d_err, coeffs ? d_err : nullptr, N, d_profile, d_cost, d_time,
+                        base + off_ws, ws_bytes, stream, true, 2);
+        if (rc != SPDY_OK) return rc;
     }
     SPDY_CUDA_TRY(cudaMemcpyAsync(profile_host, d_profile, static_cast<size_t>(N) * plan->L, cudaMemcpyDeviceToHost, stream));
     SPDY_CUDA_TRY(cudaMemcpyAsync(cost_host, d_cost, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
