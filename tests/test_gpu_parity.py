@@ -495,3 +495,34 @@ def test_byte_table_merges_equal_time_choices_only_where_exact():
     plan.check_status()
     assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), ref)
     plan.close()
+
+
+def test_random_shapes_formats_and_launch_options():
+    """Seeded fuzz over shapes (K up to 255: several mask words; times above the budget, zeros, repeats),
+    both table formats and the launch options, against the oracle."""
+    rng = np.random.default_rng(2024)
+    for trial in range(70):
+        L = int(rng.integers(1, 13))
+        K = int(rng.choice([1, 2, 3, 17, 64, 65, 130, 255]))
+        B = int(rng.choice([0, 7, 300, 1500, 4000]))
+        scale = max(1, int(B * rng.choice([0.05, 0.3, 1.2]) / max(L, 1)) + 1)
+        times = rng.integers(0, 2 * scale + 1, size=(L, K)).astype(np.int32)
+        if rng.random() < 0.5:  # sorted like real timing tables: sparser is faster, with repeats
+            times = np.sort(times, axis=1)[:, ::-1].copy()
+        if rng.random() < 0.3:
+            times[rng.integers(L), :] = 0
+        kind = trial % 3
+        if kind == 0:
+            errors = rng.lognormal(0.0, 1.0, size=(3, L, K)).astype(np.float32)
+        elif kind == 1:
+            errors = rng.choice(np.array([0, 0.25, 0.5, 1.0], np.float32), size=(3, L, K)).astype(np.float32)
+        else:
+            errors = np.sort(rng.lognormal(0.0, 1.0, size=(3, L, K)).astype(np.float32), axis=2)
+            errors[1] = -errors[1]
+        wl = W.Workload(f"fuzz-{trial}", times, errors, B)
+        ref = oracle.solve_batch(wl.errors, wl.times, wl.B)
+        options = [dict(), dict(cluster=int(rng.choice([2, 4, 8]))), dict(rows_in_global=1),
+                   dict(threads=int(rng.choice([256, 512, 1024])))]
+        for fmt in FORMATS:
+            kw = options[int(rng.integers(len(options)))]
+            assert_same(gpu_solve(wl, fmt, **kw), ref), (trial, fmt, kw)
