@@ -28,11 +28,41 @@ SM_COUNT_NOMINAL = 148
 SM_MAX_MHZ_NOMINAL = 1965.0
 CELLS_PER_CLK_PER_SM = 32.0  # one 4-byte shared-memory read per cell update, 32 banks x 4 B per clock
 
-# DRAM bytes (read + write) of the forward kernel per candidate from an ncu capture of one wave
-# (592 candidates) of the BERT-base shape; traffic grows in proportion to N.  Valid only for the
-# library version the counters were taken with.
-NCU_TRAFFIC = {"version": 1004, "workload_prefix": "bert-base-L72-K42",
-               "bytes_per_candidate": {"row_f32": 762.88e6 / 592, "arg_u8": 154.26e6 / 592}}
+# DRAM bytes (read + write) of the forward kernel from an ncu capture of one wave of the BERT-base shape:
+# kept, with the capture command and the library version it is valid for, in this file.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "forward_kernel_bert_base_dram_traffic.txt")
+
+
+def load_ncu_traffic(path: str = TRAFFIC_FILE) -> dict:
+    """`key = value` lines of the traffic record ('#' starts a comment); {} if the file is missing."""
+    out = {}
+    try:
+        for raw in open(path):
+            text = raw.split("#", 1)[0].strip()
+            if "=" in text:
+                key, value = (x.strip() for x in text.split("=", 1))
+                out[key] = value
+    except OSError:
+        pass
+    return out
+
+
+def ncu_traffic_per_launch(record: dict, library_version: int, workload_name: str, budget: int, cluster: int,
+                           table_name: str, candidates_per_launch: float):
+    """(bytes per launch or None, note).  None - said loudly - when the record was taken with another
+    library version (the kernel has changed since) or covers another workload."""
+    if not record:
+        return None, "no ncu traffic record under profiles/"
+    if int(record.get("library_version", -1)) != int(library_version):
+        return None, (f"ncu traffic record is for library version {record.get('library_version')}, this is "
+                      f"{library_version}: the kernel changed since the counters were taken; re-capture")
+    if (not workload_name.startswith(record.get("workload_prefix", "?")) or int(record.get("budget", -1)) != int(budget)
+            or cluster != 1 or f"{table_name}_bytes" not in record):
+        return None, "the ncu traffic record covers another workload or launch shape"
+    per_candidate = float(record[f"{table_name}_bytes"]) / float(record["candidates_captured"])
+    return per_candidate * candidates_per_launch, (f"ncu dram read+write of one launch over {record['candidates_captured']} "
+                                                   "candidates, scaled by the candidates of this launch "
+                                                   "(profiles/forward_kernel_bert_base_dram_traffic.txt)")
 
 
 def parse_args():
@@ -137,8 +167,10 @@ class ClockSampler:
         return out
 
 
-def oracle_baseline(wl, cpu_seconds: float) -> dict:
-    """The oracle as it stands on the host cores, on a bounded prefix of the same candidates."""
+def oracle_baseline(wl, cpu_seconds: float, gpu_outputs=None):
+    """The oracle as it stands on the host cores, on a bounded prefix of the same candidates.  Returns
+    (cpu_baseline, parity): with `gpu_outputs` = (profile, cost, time_used) as NumPy arrays, the oracle's
+    results for that prefix are compared with them bit for bit."""
     import oracle
 
     cores = host_cores()
@@ -148,11 +180,19 @@ def oracle_baseline(wl, cpu_seconds: float) -> dict:
     n = int(min(wl.N, max(cores, cpu_seconds * cores / t_one)))
     threads = min(cores, n)
     t0 = time.perf_counter()
-    oracle.solve_batch(wl.errors[:n], wl.times, wl.B, threads=threads)
+    ref = oracle.solve_batch(wl.errors[:n], wl.times, wl.B, threads=threads)
     dt = time.perf_counter() - t0
-    return {"value": n / dt, "unit": "candidates/s", "cores": threads, "kind": "oracle",
+    parity = None
+    if gpu_outputs is not None:
+        p, c, t = gpu_outputs
+        exact = bool(np.array_equal(p[:n], ref[0]) and c[:n].tobytes() == ref[1].tobytes()
+                     and np.array_equal(t[:n], ref[2]))
+        parity = {"compared": n, "of": wl.N, "bit_exact": exact,
+                  "what": "profile, fp32 cost bits and time_used of the timed launch configuration against the oracle"}
+    base = {"value": n / dt, "unit": "candidates/s", "cores": threads, "kind": "oracle",
             "sample": f"first {n} of {wl.N} candidates of {wl.name}, one single-threaded solver per core",
             "single_core_ms_per_candidate": 1e3 * t_one, "seconds": dt}
+    return base, parity
 
 
 def run_reference(args):
@@ -200,11 +240,16 @@ def run_ours(args):
 
     from paper_2201_13096_b200 import binding, sharding, workloads as W
 
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the solver has no CPU path")
+    if args.gpus > 1 and not sharding.under_launcher():
+        # Started plainly with --gpus N: start the N ranks here, one process per GPU; rank 0 prints the line.
+        if torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus} asked for, {torch.cuda.device_count()} CUDA devices visible")
+        raise SystemExit(sharding.spawn_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the solver has no CPU path")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
@@ -339,10 +384,10 @@ def run_ours(args):
     cellb = 4 if info["table_format"] == 2 else 1
     hbm_bytes = wl.N * (info["band_cells"] * cellb + wl.L * wl.K * 4)
     table_name = {1: "arg_u8", 2: "row_f32"}[info["table_format"]]
-    traffic = None
-    if (binding.library().spdy_version() == NCU_TRAFFIC["version"] and info["cluster"] == 1
-            and wl.name.startswith(NCU_TRAFFIC["workload_prefix"]) and wl.B == 10000):
-        traffic = NCU_TRAFFIC["bytes_per_candidate"][table_name] * wl.N / waves
+    traffic, traffic_note = ncu_traffic_per_launch(load_ncu_traffic(), binding.library().spdy_version(), wl.name, wl.B,
+                                                   info["cluster"], table_name, wl.N / waves)
+    if traffic is None:
+        print(f"bench.py: roofline.traffic = null: {traffic_note}", file=sys.stderr, flush=True)
     line = {
         "metric": "candidate_profiles_per_s", "value": cand_per_s, "unit": "candidates/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
@@ -363,9 +408,14 @@ def run_ours(args):
             "bound": "alu", "kernel": "spdy_forward_kernel",
             "achieved": achieved / 1e9, "peak": peak_cells / 1e9, "unit": "Gcell-updates/s",
             "frac": achieved / peak_cells, "traffic": traffic,
-            "traffic_unit": "bytes per launch (ncu dram read+write on one wave, scaled by N)",
+            "traffic_unit": "bytes per launch", "traffic_source": traffic_note,
+            "binding_unit": "shared-memory data path of the SM (32 banks x 4 B per clock): this kernel needs one 4-byte "
+                            "read of the previous row per cell update, so the ceiling is a property of the design "
+                            "(a design that re-used a read for several updates would sit under the arithmetic "
+                            "ceiling instead); no tensor cores, HBM far from binding (roofline_hbm)",
             "peak_is": f"{info['sm_count']} SMs x {sm_max:.0f} MHz x 32 four-byte shared-memory reads per clock "
                        "(one read per cell update); of nominal unit counts, max clock of measured",
+            "frac_of_arithmetic_peak": (achieved / probe[1]) if probe[1] else None,
             "peak_measured": probe[0] / 1e9, "frac_of_measured": (achieved / probe[0]) if probe[0] else None,
             "arithmetic_peak_measured": probe[1] / 1e9,
             "peak_measured_is": "spdy_probe_peaks on this device in this run: lane-consecutive 4-byte shared-memory "
@@ -401,11 +451,16 @@ def run_ours(args):
                           "dp_ms": 1e3 * res["dp_seconds"], "eval_ms": 1e3 * res["eval_seconds"], "wall_ms": 1e3 * wall,
                           "note": "synthetic loss (microseconds per call); with a real stitched-model evaluation "
                                   "the evaluations dominate, as the paper reports"}
+    parity = None
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = oracle_baseline(wl, args.cpu_seconds)
+        gpu_out = (profile.cpu().numpy(), cost.cpu().numpy(), time_used.cpu().numpy())
+        line["cpu_baseline"], parity = oracle_baseline(wl, args.cpu_seconds, gpu_out)
+        line["parity"] = parity
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+    if parity is not None and not parity["bit_exact"]:
+        raise SystemExit("the timed launch configuration disagrees with the oracle")
 
 
 SWEEP_POINTS = [  # (config, N, B override)
@@ -415,8 +470,9 @@ SWEEP_POINTS = [  # (config, N, B override)
 
 
 def run_sweep(args):
-    """Every named shape and sweep point on one GPU: device-resident timing, the oracle on a bounded
-    sample of the same candidates (timed, and compared bit for bit with the GPU's outputs)."""
+    """Every named shape and sweep point on one GPU: device-resident timing, and the oracle on the same
+    candidates (all of them up to N = 4096, a seeded sample beyond), timed and compared bit for bit with
+    the GPU's outputs."""
     import torch
 
     import oracle
@@ -457,7 +513,10 @@ def run_sweep(args):
         t0 = time.perf_counter()
         oracle.solve_batch(wl.errors[:1], wl.times, wl.B, threads=1)
         one = time.perf_counter() - t0
-        k = int(min(wl.N, max(cores, 1.5 * cores / max(one, 1e-6))))  # about 1.5 s of oracle work per point
+        # every candidate up to N = 4096; a seeded sample of 4096 at N = 65536 and of 256 at B = 10^5, where
+        # the whole batch would take the oracle minutes (its time there is extrapolated linearly in N)
+        k = wl.N if (wl.N <= 4096 and wl.B < 100000) else (256 if wl.B >= 100000 else 4096)
+        k = int(min(wl.N, k))
         sample = np.sort(np.random.default_rng(1).choice(wl.N, size=k, replace=False))
         t0 = time.perf_counter()
         ref = oracle.solve_batch(wl.errors[sample], wl.times, wl.B, threads=min(cores, k))
@@ -485,7 +544,7 @@ def run_sweep(args):
         del errors, ws
         torch.cuda.empty_cache()
     head = ("| workload | table | CTA | GPU ms | candidates/s | nominal upd/s | executed upd/s | frac | table+errors GB/s "
-            "| oracle ms (1 core) | oracle cand/s (cores) | bit-exact (sample) |")
+            "| oracle ms (1 core) | oracle cand/s (cores) | bit-exact (candidates compared) |")
     print(head, file=sys.stderr)
     print("|" + "---|" * 12, file=sys.stderr)
     for r in rows:

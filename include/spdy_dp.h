@@ -137,7 +137,9 @@ int spdy_plan_get_info(const spdy_plan *plan, spdy_plan_info *info);
  * int32 each, either may be NULL.  For an infeasible plan widths are 0. */
 int spdy_plan_get_bands(const spdy_plan *plan, int32_t *lo_host, int32_t *width_host);
 
-/* Bytes of workspace that let N candidates run as a single wave.  Any workspace of at least
+/* The walk-back table is Algorithm 1's L x (T+1) matrix (the O(L*T) memory of Section 3.2), kept per
+ * candidate and cut down to the live band of each row.
+ * Bytes of workspace that let N candidates run as a single wave.  Any workspace of at least
  * spdy_workspace_bytes(plan, 1) is accepted; a smaller-than-full one makes the batch run as
  * several waves on the stream.  Returns 0 for a null plan or N <= 0. */
 size_t spdy_workspace_bytes(const spdy_plan *plan, int64_t N);
@@ -222,8 +224,9 @@ int spdy_uniform_profile(const int32_t *times_host, int32_t L, int32_t K, int32_
                          int32_t *choice_out, int64_t *total_out);
 
 /*
- * One-shot form of the whole path: errors[N][L][K], times[L][K], budget B -> profile, cost,
- * time_used, all device pointers on the current device except nothing else.  Reads times back to
+ * One-shot form of the whole path, in the shape of the problem statement of Section 3.1 (Eq. 1: errors
+ * e_l^s, times t_l^s, budget T in, one choice per layer out): errors[N][L][K], times[L][K], budget B ->
+ * profile, cost, time_used, all device pointers on the current device.  Reads times back to
  * the host, builds a transient plan, allocates and frees its own workspace, and waits for the
  * stream before returning (synchronous).  Convenience for callers that solve once.
  */

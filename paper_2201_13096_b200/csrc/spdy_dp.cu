@@ -237,8 +237,11 @@ __device__ __forceinline__ void update_arg_pred(float (&best)[RR], float (&idxf)
 //
 // With MASKED only cells below `limit` are stored (a CTA of a cluster owns a slice of the band and
 // must not write its neighbour's cells); without it the caller guarantees room for the whole pass.
+//
+// `prev` and `cur` carry no __restrict__: with the row buffers in global memory (GROWS) the kernel itself
+// rewrites the memory behind `prev` two layers later, so those reads must stay ordinary coherent loads.
 template <int RR, int MODE, bool MASKED>
-__device__ __forceinline__ void process_span(const float *__restrict__ prev, float *__restrict__ cur,
+__device__ __forceinline__ void process_span(const float *prev, float *cur,
                                              const int2 *__restrict__ taps, const unsigned krange,
                                              const unsigned long long *__restrict__ mask, const int MW,
                                              const int s, const int lane, void *table_row,
@@ -927,11 +930,12 @@ __global__ void spdy_fill_infeasible_kernel(uint8_t *profile, float *cost, int32
                                             int64_t N, int32_t L)
 {
     const int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     const int64_t total = N * L;
-    for (int64_t j = i; j < total; j += static_cast<int64_t>(gridDim.x) * blockDim.x) profile[j] = 0xFF;
-    if (i < N) {
-        cost[i] = pos_inf();
-        time_used[i] = -1;
+    for (int64_t j = i; j < total; j += stride) profile[j] = 0xFF;
+    for (int64_t j = i; j < N; j += stride) {
+        cost[j] = pos_inf();
+        time_used[j] = -1;
     }
 }
 
@@ -1377,8 +1381,10 @@ int choose_cluster_shape(spdy_plan *p, const spdy_options *opts, int64_t smem_pe
             if (!p->cvariant) return SPDY_ERR_INVALID_ARG;
             p->ctas_per_sm = 1;
             if (p->device >= 0) {
+                // The limit belongs to the kernel on the device, not to this plan: always the device's
+                // opt-in maximum, so that plans of different widths can live side by side.
                 SPDY_CUDA_TRY(cudaFuncSetAttribute(p->cvariant->fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   static_cast<int>(p->smem_bytes)));
+                                                   static_cast<int>(smem_per_block)));
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3(static_cast<unsigned>(C), 1, 1);
                 cfg.blockDim = dim3(static_cast<unsigned>(threads), 1, 1);
@@ -1500,8 +1506,10 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
     const int64_t by_smem = std::max<int64_t>(1, smem_per_sm / (p->smem_bytes + 1024));
     p->ctas_per_sm = static_cast<int>(std::min<int64_t>(by_smem, 2048 / best_threads));
     if (p->device >= 0) {
+        // The limit belongs to the kernel on the device, not to this plan: always the device's opt-in
+        // maximum (every plan writes the same value), so that plans of different widths can live side by side.
         SPDY_CUDA_TRY(cudaFuncSetAttribute(p->variant->fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           static_cast<int>(p->smem_bytes)));
+                                           static_cast<int>(smem_per_block)));
         int occ = 0;
         SPDY_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, p->variant->fn, best_threads,
                                                                     static_cast<size_t>(p->smem_bytes)));
@@ -1611,7 +1619,7 @@ struct DeviceGuard {
 
 extern "C" {
 
-int spdy_version(void) { return 1004; }
+int spdy_version(void) { return 1005; }
 
 int spdy_last_cuda_error(void) { return g_last_cuda_error; }
 
@@ -2053,67 +2061,76 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
     // to solve.  Every chunk boundary costs a launch tail (and a walk back, unless one serves all), so
     // chunks are few - one wave, then the rest, measured best at the BERT-base shape - and coefficient
     // input (K times smaller) goes up in one piece.
-    const int64_t per_cand = static_cast<int64_t>(plan->L) * (coeffs ? 1 : plan->K);
-    std::vector<int64_t> bounds(1, 0);
-    {
-        int64_t size = std::max<int64_t>(1, static_cast<int64_t>(plan->ctas_per_sm) * plan->sm_count / std::max(1, plan->cluster));
-        if (coeffs) size = N;
-        while (bounds.back() < N) {
-            bounds.push_back(std::min<int64_t>(N, bounds.back() + size));
-            size *= 6;
+    // Everything from the first queued copy on runs inside `enqueue`: whatever makes it stop early, the
+    // copies already queued still read the caller's host buffer, so every exit below waits for both
+    // streams before the error goes back to the caller (who may free or reuse the buffer on seeing it).
+    auto enqueue = [&]() -> int {
+        const int64_t per_cand = static_cast<int64_t>(plan->L) * (coeffs ? 1 : plan->K);
+        std::vector<int64_t> bounds(1, 0);
+        {
+            int64_t size = std::max<int64_t>(1, static_cast<int64_t>(plan->ctas_per_sm) * plan->sm_count / std::max(1, plan->cluster));
+            if (coeffs) size = N;
+            while (bounds.back() < N) {
+                bounds.push_back(std::min<int64_t>(N, bounds.back() + size));
+                size *= 6;
+            }
         }
-    }
-    const size_t chunks = bounds.size() - 1;
-    if (chunks > 1) {
-        if (!plan->copy_stream) SPDY_CUDA_TRY(cudaStreamCreateWithFlags(&plan->copy_stream, cudaStreamNonBlocking));
-        if (!plan->entry_event) SPDY_CUDA_TRY(cudaEventCreateWithFlags(&plan->entry_event, cudaEventDisableTiming));
-        while (plan->copy_events.size() < chunks) {
-            cudaEvent_t e;
-            SPDY_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-            plan->copy_events.push_back(e);
+        const size_t chunks = bounds.size() - 1;
+        if (chunks > 1) {
+            if (!plan->copy_stream) SPDY_CUDA_TRY(cudaStreamCreateWithFlags(&plan->copy_stream, cudaStreamNonBlocking));
+            if (!plan->entry_event) SPDY_CUDA_TRY(cudaEventCreateWithFlags(&plan->entry_event, cudaEventDisableTiming));
+            while (plan->copy_events.size() < chunks) {
+                cudaEvent_t e;
+                SPDY_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+                plan->copy_events.push_back(e);
+            }
+            // Work already queued on the caller's stream may still read the staging buffer.
+            SPDY_CUDA_TRY(cudaEventRecord(plan->entry_event, stream));
+            SPDY_CUDA_TRY(cudaStreamWaitEvent(plan->copy_stream, plan->entry_event, 0));
+            for (size_t c = 0; c < chunks; ++c) {
+                const int64_t first = bounds[c], count = bounds[c + 1] - bounds[c];
+                SPDY_CUDA_TRY(cudaMemcpyAsync(d_err + first * per_cand, errors_host + first * per_cand,
+                                              static_cast<size_t>(count * per_cand) * sizeof(float),
+                                              cudaMemcpyHostToDevice, plan->copy_stream));
+                SPDY_CUDA_TRY(cudaEventRecord(plan->copy_events[c], plan->copy_stream));
+            }
+        } else {
+            SPDY_CUDA_TRY(cudaMemcpyAsync(d_err, errors_host, err_bytes, cudaMemcpyHostToDevice, stream));
         }
-        // Work already queued on the caller's stream may still read the staging buffer.
-        SPDY_CUDA_TRY(cudaEventRecord(plan->entry_event, stream));
-        SPDY_CUDA_TRY(cudaStreamWaitEvent(plan->copy_stream, plan->entry_event, 0));
+        // When the whole batch's table fits the staging workspace (and nothing but tables lives there),
+        // the chunks' forward passes write disjoint parts of it and ONE walk back follows: the walk back
+        // is a latency chain of L steps whatever the number of candidates.
+        const bool one_walk_back = chunks > 1 && plan->feasible && !plan->merged && !plan->global_rows &&
+                                   ws_bytes >= ws_one * static_cast<size_t>(N);
         for (size_t c = 0; c < chunks; ++c) {
             const int64_t first = bounds[c], count = bounds[c + 1] - bounds[c];
-            SPDY_CUDA_TRY(cudaMemcpyAsync(d_err + first * per_cand, errors_host + first * per_cand,
-                                          static_cast<size_t>(count * per_cand) * sizeof(float),
-                                          cudaMemcpyHostToDevice, plan->copy_stream));
-            SPDY_CUDA_TRY(cudaEventRecord(plan->copy_events[c], plan->copy_stream));
+            if (chunks > 1) SPDY_CUDA_TRY(cudaStreamWaitEvent(stream, plan->copy_events[c], 0));
+            const float *in = d_err + first * per_cand;
+            if (one_walk_back)
+                rc = solve_impl(plan, coeffs ? nullptr : in, coeffs ? in : nullptr, count, d_profile + first * plan->L,
+                                d_cost + first, d_time + first, base + off_ws + static_cast<size_t>(first) * ws_one,
+                                static_cast<size_t>(count) * ws_one, stream, c > 0, 1);
+            else
+                rc = solve_impl(plan, coeffs ? nullptr : in, coeffs ? in : nullptr, count, d_profile + first * plan->L,
+                                d_cost + first, d_time + first, base + off_ws, ws_bytes, stream, c > 0);
+            if (rc != SPDY_OK) return rc;
         }
-    } else {
-        SPDY_CUDA_TRY(cudaMemcpyAsync(d_err, errors_host, err_bytes, cudaMemcpyHostToDevice, stream));
-    }
-    // When the whole batch's table fits the staging workspace (and nothing but tables lives there),
-    // the chunks' forward passes write disjoint parts of it and ONE walk back follows: the walk back
-    // is a latency chain of L steps whatever the number of candidates.
-    const bool one_walk_back = chunks > 1 && plan->feasible && !plan->merged && !plan->global_rows &&
-                               ws_bytes >= ws_one * static_cast<size_t>(N);
-    for (size_t c = 0; c < chunks; ++c) {
-        const int64_t first = bounds[c], count = bounds[c + 1] - bounds[c];
-        if (chunks > 1) SPDY_CUDA_TRY(cudaStreamWaitEvent(stream, plan->copy_events[c], 0));
-        const float *in = d_err + first * per_cand;
-        if (one_walk_back)
-            rc = solve_impl(plan, coeffs ? nullptr : in, coeffs ? in : nullptr, count, d_profile + first * plan->L,
-                            d_cost + first, d_time + first, base + off_ws + static_cast<size_t>(first) * ws_one,
-                            static_cast<size_t>(count) * ws_one, stream, c > 0, 1);
-        else
-            rc = solve_impl(plan, coeffs ? nullptr : in, coeffs ? in : nullptr, count, d_profile + first * plan->L,
-                            d_cost + first, d_time + first, base + off_ws, ws_bytes, stream, c > 0);
-        if (rc != SPDY_OK) {
-            if (chunks > 1) cudaStreamSynchronize(plan->copy_stream);
-            return rc;
+        if (one_walk_back) {
+            rc = solve_impl(plan, coeffs ? nullptr : d_err, coeffs ? d_err : nullptr, N, d_profile, d_cost, d_time,
+                            base + off_ws, ws_bytes, stream, true, 2);
+            if (rc != SPDY_OK) return rc;
         }
+        SPDY_CUDA_TRY(cudaMemcpyAsync(profile_host, d_profile, static_cast<size_t>(N) * plan->L, cudaMemcpyDeviceToHost, stream));
+        SPDY_CUDA_TRY(cudaMemcpyAsync(cost_host, d_cost, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
+        SPDY_CUDA_TRY(cudaMemcpyAsync(time_used_host, d_time, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
+        return SPDY_OK;
+    };
+    rc = enqueue();
+    if (rc != SPDY_OK) {
+        if (plan->copy_stream) cudaStreamSynchronize(plan->copy_stream);
+        cudaStreamSynchronize(stream);
+        return rc;
     }
-    if (one_walk_back) {
-        rc = solve_impl(plan, coeffs ? nullptr : d_err, coeffs ? d_err : nullptr, N, d_profile, d_cost, d_time,
-                        base + off_ws, ws_bytes, stream, true, 2);
-        if (rc != SPDY_OK) return rc;
-    }
-    SPDY_CUDA_TRY(cudaMemcpyAsync(profile_host, d_profile, static_cast<size_t>(N) * plan->L, cudaMemcpyDeviceToHost, stream));
-    SPDY_CUDA_TRY(cudaMemcpyAsync(cost_host, d_cost, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
-    SPDY_CUDA_TRY(cudaMemcpyAsync(time_used_host, d_time, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
     SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
     return SPDY_OK;
 }

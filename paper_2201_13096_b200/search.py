@@ -1,4 +1,4 @@
-"""SPDY's search for sensitivity coefficients (Section 3.3; Appendix A, Algorithm 4) with the dynamic
+"""SPDY's search for sensitivity coefficients (Section 3.3; Appendix B, Algorithm 4) with the dynamic
 programs of many trials solved in one GPU batch.
 
 Algorithm 4 is sequential: every trial mutates the current best vector c* and replaces it when the

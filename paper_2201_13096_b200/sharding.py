@@ -3,7 +3,11 @@ so the path shards with no data-path collective: each rank solves a contiguous s
 exchanges are control-plane: a barrier and a MAX reduction of timings."""
 from __future__ import annotations
 
-from typing import Tuple
+import os
+import socket
+import subprocess
+import sys
+from typing import List, Optional, Sequence, Tuple
 
 
 def shard_range(n_total: int, rank: int, world: int) -> Tuple[int, int]:
@@ -33,3 +37,33 @@ def whole_job_rate(units_per_rank: int, world: int, seconds_max: float) -> float
     """Aggregate throughput when every rank processed ``units_per_rank`` units (weak scaling) and
     the slowest rank took ``seconds_max``."""
     return world * units_per_rank / seconds_max
+
+
+def free_port() -> int:
+    """A TCP port on 127.0.0.1 that is free right now (for the rendezvous of a local launch)."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return int(s.getsockname()[1])
+
+
+def launch_command(script: str, script_args: Sequence[str], nproc: int, port: Optional[int] = None) -> List[str]:
+    """The command that starts ``nproc`` ranks of ``script`` on this node, one process per rank, with a
+    127.0.0.1 rendezvous (the container's hostname may not resolve)."""
+    if nproc < 1:
+        raise ValueError("need at least one rank")
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={int(nproc)}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port if port is not None else free_port()),
+            script, *script_args]
+
+
+def under_launcher() -> bool:
+    """True inside a process that a launcher started as one rank of several (WORLD_SIZE is set)."""
+    return "WORLD_SIZE" in os.environ
+
+
+def spawn_ranks(script: str, script_args: Sequence[str], nproc: int, timeout: Optional[float] = None) -> int:
+    """Run ``script`` as ``nproc`` ranks and wait; the ranks inherit stdout/stderr (rank 0 prints the
+    result).  Returns the launcher's exit code."""
+    env = dict(os.environ)
+    env.setdefault("OMP_NUM_THREADS", "1")
+    return subprocess.run(launch_command(script, script_args, nproc), env=env, timeout=timeout).returncode

@@ -7,7 +7,6 @@ import pytest
 
 import oracle
 from paper_2201_13096_b200 import binding, build as build_mod, workloads as W
-from helpers import check_solution
 
 pytestmark = pytest.mark.gpu
 
@@ -170,11 +169,25 @@ def test_host_buffer_and_one_shot_entry_points():
     assert (p.cpu().numpy() == 0xFF).all() and (t.cpu().numpy() == -1).all() and np.isposinf(c.cpu().numpy()).all()
 
 
-def check_full_size(wl, sample_size, fmt=0, workspace_bytes=None):
-    """Invariants that hold at any size on every candidate, and the oracle on a seeded sample."""
+_ORACLE_CACHE = {}
+
+
+def oracle_on(wl, key, sample=None):
+    """Oracle outputs for the candidates `sample` (all when None) of a named workload, computed once per
+    test session: the table formats and launch options under test share them."""
+    if key not in _ORACLE_CACHE:
+        errors = wl.errors if sample is None else wl.errors[sample]
+        _ORACLE_CACHE[key] = oracle.solve_batch(errors, wl.times, wl.B, threads=CORES)
+    return _ORACLE_CACHE[key]
+
+
+def check_full_size(wl, key, sample_size=None, fmt=0, workspace_bytes=None, **plan_kw):
+    """A batch at its full size, in the launch shape the plan picks by default: every candidate against the
+    oracle (`sample_size` None), or - where the oracle would take minutes - a seeded sample of that size
+    against the oracle and, on every candidate, the invariants that hold at any size."""
     import torch
 
-    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt, **plan_kw)
     ws = None
     if workspace_bytes is not None:
         per = plan.workspace_bytes(1)
@@ -185,6 +198,9 @@ def check_full_size(wl, sample_size, fmt=0, workspace_bytes=None):
     p, c, t = p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()
     del ws
     plan.close()
+    if sample_size is None:
+        assert_same((p, c, t), oracle_on(wl, key))
+        return
     assert (t >= 0).all() and (t <= wl.B).all() and (p < wl.K).all()
     idx = p.astype(np.int64)
     assert np.array_equal(wl.times[np.arange(wl.L)[None, :], idx].sum(axis=1), t)
@@ -194,50 +210,47 @@ def check_full_size(wl, sample_size, fmt=0, workspace_bytes=None):
         acc = (acc + e_sel[:, l]).astype(np.float32)
     assert acc.tobytes() == c.tobytes()
     sample = np.sort(np.random.default_rng(0).choice(wl.N, size=min(sample_size, wl.N), replace=False))
-    ref = oracle.solve_batch(wl.errors[sample], wl.times, wl.B, threads=CORES)
-    assert_same((p[sample], c[sample], t[sample]), ref)
+    assert_same((p[sample], c[sample], t[sample]), oracle_on(wl, (key, sample_size), sample))
 
 
 @pytest.mark.parametrize("fmt", FORMATS)
-def test_full_size_resnet50_and_bert_large_batches(fmt):
-    """Configs 1 and 3 at their full N = 1024, in the launch shape the plan picks by default."""
-    check_full_size(W.make_workload(1), 96, fmt)
-    check_full_size(W.make_workload(3), 8, fmt)
+def test_full_size_resnet50_batch_every_candidate(fmt):
+    """Config 1 at its full N = 1024, every candidate against the oracle."""
+    check_full_size(W.make_workload(1), "cfg1", fmt=fmt)
 
 
-def test_full_size_sweep_points():
-    """Config 4's largest points: N = 65536 (run in waves inside a 12 GB workspace) and B = 100000."""
-    check_full_size(W.make_workload(4, N=65536), 64, workspace_bytes=12 << 30)
-    check_full_size(W.make_workload(4, N=4096, B=1000), 256)
-    check_full_size(W.make_workload(4, N=1024, B=100000), 6)
-
-
-def test_full_size_bert_base_batch_in_the_benchmark_configuration():
-    """N = 4096 as the benchmark times it: invariants on every candidate, oracle on a sample."""
-    import torch
-
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_full_size_bert_base_batch_every_candidate_in_the_benchmark_configuration(fmt):
+    """Config 2, N = 4096, as the benchmark times it (default plan, one wave): every candidate's profile,
+    cost bits and time_used against the oracle."""
     wl = W.make_workload(2)
     assert wl.N == 4096
-    plan = binding.Plan(wl.times, wl.B, device=0)
-    p, c, t = binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda())
-    torch.cuda.synchronize()
-    plan.check_status()
-    p, c, t = p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()
-    # invariants at full size (vectorised): total time and left-to-right fp32 sum of the profile
-    assert (t >= 0).all() and (t <= wl.B).all() and (p < wl.K).all()
-    idx = p.astype(np.int64)
-    tt = wl.times[np.arange(wl.L)[None, :], idx].sum(axis=1)
-    assert np.array_equal(tt, t)
-    e_sel = np.take_along_axis(wl.errors, idx[:, :, None], axis=2)[:, :, 0]
-    acc = np.zeros(wl.N, np.float32)
-    for l in range(wl.L):
-        acc = (acc + e_sel[:, l]).astype(np.float32)
-    assert acc.tobytes() == c.tobytes()
-    sample = np.random.default_rng(0).choice(wl.N, size=64, replace=False)
-    ref = oracle.solve_batch(wl.errors[sample], wl.times, wl.B, threads=CORES)
-    assert_same((p[sample], c[sample], t[sample]), ref)
-    for n in sample[:4]:
-        check_solution(wl.errors[n], wl.times, wl.B, p[n], c[n], int(t[n]))
+    check_full_size(wl, "cfg2", fmt=fmt)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_full_size_bert_large_batch_every_candidate(fmt):
+    """Config 3 at its full N = 1024 (B = 65536, K = 64), every candidate against the oracle."""
+    check_full_size(W.make_workload(3), "cfg3", fmt=fmt)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_full_size_sweep_points(fmt):
+    """Config 4's largest points.  N = 65536 runs in waves inside a 12 GB workspace and is compared with the
+    oracle on 4096 seeded candidates; B = 1000 on all 4096; B = 100000 (rows in global memory) on 256 of
+    1024.  The sampled points also get the any-size invariants on every candidate."""
+    check_full_size(W.make_workload(4, N=65536), "N65536", 4096, fmt=fmt, workspace_bytes=12 << 30)
+    check_full_size(W.make_workload(4, N=4096, B=1000), "B1000", fmt=fmt)
+    check_full_size(W.make_workload(4, N=1024, B=100000), "B100000", 256, fmt=fmt)
+
+
+def test_sweep_points_with_few_candidates_every_candidate():
+    """Config 4's small batches (N = 1, 16, 256), every candidate, both table formats."""
+    for n in (1, 16, 256):
+        wl = W.make_workload(4, N=n)
+        ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+        for fmt in FORMATS:
+            assert_same(gpu_solve(wl, fmt), ref)
 
 
 @pytest.mark.parametrize("cluster", [2, 4, 8])
@@ -407,8 +420,7 @@ def test_host_buffer_path_uploads_in_chunks():
     for errors in (wl.errors, pinned, wl.errors[:700], wl.errors):
         n = len(errors)
         assert_same(binding.solve_batch_host(plan, errors), tuple(x[:n] for x in dev))
-    sample = np.arange(0, 2500, 97)
-    assert_same(tuple(x[sample] for x in dev), oracle.solve_batch(wl.errors[sample], wl.times, wl.B, threads=CORES))
+    assert_same(dev, oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
     coeffs = W.sensitivity_samples(3, wl.L, 2500)
     pc, cc, tc = binding.solve_batch_coeffs(plan, torch.from_numpy(coeffs).cuda())
     torch.cuda.synchronize()
@@ -526,3 +538,44 @@ def test_random_shapes_formats_and_launch_options():
         for fmt in FORMATS:
             kw = options[int(rng.integers(len(options)))]
             assert_same(gpu_solve(wl, fmt, **kw), ref), (trial, fmt, kw)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_two_live_plans_of_one_kernel_variant(fmt):
+    """A wide plan (more than 48 KB of dynamic shared memory per CTA) must keep working after a narrower
+    plan of the same table format and CTA size has been created, and after a call of the static entry
+    point: the shared-memory limit is a property of the kernel on the device, not of a plan."""
+    import torch
+
+    wide = W.make_workload(2, N=12)
+    narrow = W.make_workload(4, N=12, B=2500)
+    ref_wide = oracle.solve_batch(wide.errors, wide.times, wide.B, threads=CORES)
+    ref_narrow = oracle.solve_batch(narrow.errors, narrow.times, narrow.B, threads=CORES)
+    for between in (False, True):
+        a = binding.Plan(wide.times, wide.B, device=0, table_format=fmt, threads=128)
+        b = binding.Plan(narrow.times, narrow.B, device=0, table_format=fmt, threads=128)
+        assert a.info["smem_bytes"] > 48 * 1024 > b.info["smem_bytes"]
+        if between:
+            binding.solve_batch_static(torch.from_numpy(narrow.errors).cuda(), narrow.times, narrow.B)
+        for plan, wl, ref in ((a, wide, ref_wide), (b, narrow, ref_narrow), (a, wide, ref_wide)):
+            p, c, t = binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda())
+            torch.cuda.synchronize()
+            plan.check_status()
+            assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), ref)
+        a.close()
+        b.close()
+
+
+def test_plan_level_infeasible_budget_fills_every_candidate():
+    """The marker outputs of an infeasible plan reach every candidate, also of a batch with more
+    candidates than 65535 blocks of 256 threads."""
+    import torch
+
+    times = np.array([[5, 6], [7, 9]], np.int32)
+    N = 65535 * 256 + 999
+    plan = binding.Plan(times, 11, device=0)
+    assert plan.info["feasible"] == 0
+    p, c, t = binding.solve_batch(plan, torch.empty((N, 2, 2), device="cuda"))
+    torch.cuda.synchronize()
+    assert (p == 0xFF).all().item() and (t == -1).all().item() and torch.isposinf(c).all().item()
+    plan.close()

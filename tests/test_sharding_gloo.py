@@ -1,8 +1,10 @@
 """The N>1 path on CPU: two gloo ranks shard one candidate stream, solve their slices (with the
 CPU oracle standing in for the device here), and agree on max-over-ranks timing; the union of the
 shards must equal the unsharded batch."""
+import json
 import os
 import socket
+import subprocess
 
 import numpy as np
 import torch
@@ -66,3 +68,20 @@ def test_two_gloo_ranks_cover_the_batch(tmp_path):
 def test_max_over_ranks_without_a_process_group():
     assert sharding.max_over_ranks(3.5) == 3.5
     assert sharding.whole_job_rate(100, 4, 2.0) == 200.0
+
+
+def test_local_launcher_starts_the_ranks_itself():
+    """The launch path `bench.py --gpus N` takes when no launcher started it: N ranks on this node with
+    a 127.0.0.1 rendezvous, rank 0 printing the line.  Here with two gloo ranks on CPU."""
+    script = os.path.join(os.path.dirname(os.path.abspath(__file__)), "rank_probe.py")
+    cmd = sharding.launch_command(script, ["11"], 2)
+    assert "--master-addr" in cmd and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    out = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads([ln for ln in out.stdout.splitlines() if ln.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["worst"] == 2.0
+    assert line["shards"] == [[0, 6], [6, 5]]
+    assert not sharding.under_launcher() or "WORLD_SIZE" in os.environ
+    with __import__("pytest").raises(ValueError):
+        sharding.launch_command(script, [], 0)

@@ -3,14 +3,17 @@
 Some users of this library run where a device allocation is off limits: inside a framework that
 owns the whole device heap, or in a service whose memory footprint is frozen after start-up.
 ``spdy_solve_batch_static`` serves them from an array compiled into the library.  This file checks
-it, through the C ABI, against the ordinary entry point - twice in a row, because the array keeps
-the first call's leftovers when the second one starts.  It is collected last on purpose.
+it, through the C ABI, against the ordinary entry point and against the CPU oracle - twice in a row,
+because the array keeps the first call's leftovers when the second one starts.  It is collected last
+on purpose.
 """
 import ctypes
+import os
 
 import numpy as np
 import pytest
 
+import oracle
 from paper_2201_13096_b200 import binding, build as build_mod, workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -50,6 +53,10 @@ def test_static_scratch_entry_point_matches_the_allocating_one_twice_in_a_row():
         assert torch.equal(time_used, want_t)
         assert cost.cpu().numpy().tobytes() == want_c.cpu().numpy().tobytes()
         plan.close()
+        # and both agree with the oracle, element by element
+        rp, rc_, rt = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=max(1, len(os.sched_getaffinity(0))))
+        assert np.array_equal(profile.cpu().numpy(), rp) and np.array_equal(time_used.cpu().numpy(), rt)
+        assert cost.cpu().numpy().tobytes() == rc_.tobytes()
 
 
 def test_static_entry_point_rejects_what_does_not_fit():
