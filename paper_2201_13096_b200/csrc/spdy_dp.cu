@@ -1383,8 +1383,10 @@ int choose_cluster_shape(spdy_plan *p, const spdy_options *opts, int64_t smem_pe
             if (p->device >= 0) {
                 // The limit belongs to the kernel on the device, not to this plan: always the device's
                 // opt-in maximum, so that plans of different widths can live side by side.
+                cudaFuncAttributes fattr;
+                SPDY_CUDA_TRY(cudaFuncGetAttributes(&fattr, p->cvariant->fn));
                 SPDY_CUDA_TRY(cudaFuncSetAttribute(p->cvariant->fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   static_cast<int>(smem_per_block)));
+                                                   static_cast<int>(smem_per_block - static_cast<int64_t>(fattr.sharedSizeBytes))));
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3(static_cast<unsigned>(C), 1, 1);
                 cfg.blockDim = dim3(static_cast<unsigned>(threads), 1, 1);
@@ -1507,9 +1509,11 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
     p->ctas_per_sm = static_cast<int>(std::min<int64_t>(by_smem, 2048 / best_threads));
     if (p->device >= 0) {
         // The limit belongs to the kernel on the device, not to this plan: always the device's opt-in
-        // maximum (every plan writes the same value), so that plans of different widths can live side by side.
+        // maximum less the kernel's static shared memory (every plan writes the same value), so that plans of different widths can live side by side.
+        cudaFuncAttributes fattr;
+        SPDY_CUDA_TRY(cudaFuncGetAttributes(&fattr, p->variant->fn));
         SPDY_CUDA_TRY(cudaFuncSetAttribute(p->variant->fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           static_cast<int>(smem_per_block)));
+                                           static_cast<int>(smem_per_block - static_cast<int64_t>(fattr.sharedSizeBytes))));
         int occ = 0;
         SPDY_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, p->variant->fn, best_threads,
                                                                     static_cast<size_t>(p->smem_bytes)));
