@@ -45,7 +45,8 @@ typedef enum spdy_status {
     SPDY_ERR_CUDA = -4,               /* a CUDA runtime call failed; see spdy_last_cuda_error() */
     SPDY_ERR_NO_MEMORY = -5,          /* host or device allocation failed */
     SPDY_ERR_INTERNAL = -6,           /* a self-check inside the kernels failed */
-    SPDY_ERR_STATIC_LIMIT = -7        /* spdy_solve_batch_static: problem exceeds its built-in scratch */
+    SPDY_ERR_STATIC_LIMIT = -7,       /* spdy_solve_batch_static: problem exceeds its built-in scratch */
+    SPDY_ERR_NO_DEVICE_CODE = -8      /* a device was asked of the host-only build of the library */
 } spdy_status;
 
 /*
@@ -68,22 +69,38 @@ typedef enum spdy_table_format {
     SPDY_TABLE_ROW_F32 = 2
 } spdy_table_format;
 
+/* Which kernel family runs the forward pass when one CTA-sized unit works on a candidate. */
+typedef enum spdy_kernel {
+    SPDY_KERNEL_AUTO = 0, /* let the plan choose */
+    SPDY_KERNEL_CTA = 1,  /* one CTA per candidate, one block barrier per layer */
+    SPDY_KERNEL_WARP = 2  /* one warp per candidate, four candidates per CTA, no block barrier: for rows a
+                             warp pass or two wide (a budget of about a thousand buckets) */
+} spdy_kernel;
+
 typedef struct spdy_options {
     int32_t table_format;  /* spdy_table_format */
     int32_t threads;       /* threads per CTA, 0 = choose; one of 128, 256, 512, 1024 and >= K */
-    int32_t cluster;       /* CTAs cooperating on one candidate: 0 or 1 = one CTA (the default); 2, 4 or 8 = a
+    int32_t cluster;       /* CTAs cooperating on one candidate: 0 = choose, 1 = one CTA; 2, 4 or 8 = a
                               thread-block cluster that splits every row, which shortens the latency of
                               batches with fewer candidates than SMs.  1 also forbids the fallbacks for
                               rows too wide for one CTA's shared memory (UNSUPPORTED instead) */
     int32_t forward_mode;  /* 0 = choose.  Variants of the forward kernel's cell update, all with
                               identical results, for measurement: 1 compare+select (ARG_U8),
                               2 compare+predicated moves (ARG_U8), 3 fp32 minimum (ROW_F32),
-                              4 packed adds + 3-input minimum over choice pairs (ROW_F32) */
+                              4 packed adds + 3-input minimum over slot pairs (ROW_F32),
+                              5 3-input minimum over slot pairs, index resolved from the outcome (ARG_U8) */
     int32_t rows_in_global; /* 1: keep the two dynamic-program rows in the workspace (global memory) rather than
                               in shared memory and read them through L1.  Chosen automatically when two rows
                               do not fit one CTA's shared memory (B of about 10^5 buckets and more); any width
                               runs.  One CTA of 1024 threads per candidate; not combinable with cluster > 1 */
-    int32_t reserved[3];   /* must be 0 */
+    int32_t kernel;        /* spdy_kernel */
+    int32_t schedule;      /* how a row is cut into warp passes.  Bits 0-7: 0 = passes sized by the slots that
+                              overlap them and dealt to the warps by cost (default), 1 = passes of one size dealt
+                              round-robin (for measurement).  Bits 8-15: upper limit of cells per lane per pass,
+                              1..24 (0 = the kernel's own limit; for measurement) */
+    int32_t auto_shape;    /* 0: when threads, cluster, rows_in_global and kernel are all 0 the plan also lays
+                              out launch shapes for batches too small to fill the device (larger CTAs, clusters
+                              of 2/4/8) and spdy_solve_batch picks by N; 1: never, one shape for every N */
 } spdy_options;
 
 /* Facts about a plan: shapes, the launch shape chosen, and work counts for measurement. */
@@ -109,6 +126,10 @@ typedef struct spdy_plan_info {
                                  byte table this is the count for candidates that may be merged (see
                                  spdy_table_format); issued_updates is given for the same table set */
     int32_t launches_per_wave; /* kernels one wave of candidates launches (2, or 5 with the byte table's two table sets) */
+    int32_t kernel;            /* spdy_kernel of the main launch shape (CTA also for clusters and rows in global memory) */
+    int32_t forward_mode;      /* resolved cell-update variant (see spdy_options.forward_mode) */
+    int32_t candidates_per_cta;/* 1, or 4 with one warp per candidate */
+    int32_t alternates;        /* further launch shapes laid out for small batches (see spdy_options.auto_shape) */
     int32_t reserved1;
 } spdy_plan_info;
 
@@ -120,7 +141,8 @@ typedef struct spdy_plan spdy_plan; /* opaque; owns only its own small host and 
  * one small host-to-device copy on `device`.
  *   times_host  host, [L][K] int32 row-major, read during the call only.
  *   device      CUDA device ordinal, or -1 for a host-only plan (info queries only; solving
- *               with it returns SPDY_ERR_INVALID_ARG).
+ *               with it returns SPDY_ERR_INVALID_ARG).  The host-only build of the library
+ *               (libspdy_plan_host.so: plans, helpers, no kernels) accepts -1 only.
  *   opts        host, may be NULL for defaults.
  *   *out        receives the plan; destroy with spdy_plan_destroy.
  * Errors: INVALID_ARG (null, L<1, K<1, K>255, B<0, a negative time, bad option), UNSUPPORTED
@@ -136,6 +158,46 @@ int spdy_plan_get_info(const spdy_plan *plan, spdy_plan_info *info);
 /* Per-layer live band [lo, lo+width) of row l (l = 1..L stored at index l-1); host arrays of L
  * int32 each, either may be NULL.  For an infeasible plan widths are 0. */
 int spdy_plan_get_bands(const spdy_plan *plan, int32_t *lo_host, int32_t *width_host);
+
+/*
+ * Inspection of a plan's host tables, for tests and tools (no GPU work).  `which` selects the table set:
+ * 0 = the main launch shape, -1 = the byte table's second set with merged equal-time choices (INVALID_ARG
+ * if there is none), i >= 1 = the i-th launch shape for small batches.  The pointers stay valid until the
+ * plan is destroyed.
+ *   layers      [L][8] int32: width, row offset in the table, lo, smallest usable time, extent (cells the
+ *               passes write, a multiple of 32), shift slots, 0, 0
+ *   slots       [L][K][2] int32: (a, b) of each shift slot: it contributes to band cells a..b and reads the
+ *               previous row at cell - a (the first layers[l][5] entries of a layer are valid)
+ *   passes      [n_passes][2]: first cell, and u_lo | u_hi << 8 | dense << 16 | cells_per_lane << 24
+ *   pass_masks  [n_passes][mask_words] uint64: bit u set = slot u overlaps the pass
+ *   pass_ptr    [L * warps_per_candidate + 1]: the passes of (layer l, warp w) are pass_ptr[l*W+w] ..
+ *               pass_ptr[l*W+w+1] (NULL for a cluster shape, whose passes are listed per slice)
+ *   slices      [L][cluster][8] int32 for a cluster shape (slice_lo, slice_hi, cells per lane, passes, first
+ *               pass, first window cell, window length, slice length of the previous row), else NULL
+ * spdy_plan_verify re-derives on the host, for every layer, pass and slot of every table set of the plan, the
+ * lowest and highest row-buffer cell a lane reads and the cells it writes, and checks them against the
+ * buffers' extents and against the region known to hold the previous row or +inf (Algorithm 1's shifted
+ * read D[l-1, t - t_l^s]): SPDY_OK, or SPDY_ERR_INTERNAL on the first violation.  Every plan is verified
+ * this way when it is created.
+ */
+typedef struct spdy_plan_tables {
+    int32_t L, K;
+    int32_t kernel_kind;         /* 0 CTA per candidate, 1 CTA with rows in global memory, 2 cluster, 3 warp per candidate */
+    int32_t threads, warps_per_candidate, cluster, forward_mode;
+    int32_t max_cells_per_lane;  /* the kernel build's largest pass */
+    int32_t row_stride, pad;     /* floats per row buffer; guard cells of +inf on either side of a row */
+    int32_t out_stride, win_stride; /* cluster shape: floats per slice buffer and per window */
+    int32_t mask_words, n_passes;
+    int64_t pitch;               /* table cells per candidate */
+    const int32_t *layers;
+    const int32_t *slots;
+    const int32_t *passes;
+    const uint64_t *pass_masks;
+    const int32_t *pass_ptr;
+    const int32_t *slices;
+} spdy_plan_tables;
+int spdy_plan_get_tables(const spdy_plan *plan, int32_t which, spdy_plan_tables *out);
+int spdy_plan_verify(const spdy_plan *plan);
 
 /* The walk-back table is Algorithm 1's L x (T+1) matrix (the O(L*T) memory of Section 3.2), kept per
  * candidate and cut down to the live band of each row.
@@ -241,6 +303,18 @@ int spdy_solve_batch_simple(const float *errors_dev, const int32_t *times_dev, i
  * SPDY_ERR_INTERNAL if the word was set, or a CUDA error.
  */
 int spdy_plan_check_status(spdy_plan *plan, void *cuda_stream);
+
+/*
+ * The same word, returned rather than judged: *word_host receives it (0 = nothing flagged) and it is
+ * cleared.  Bit 0: the walk back met an invalid table entry.  The remaining bits are set only by the debug
+ * build of the library (libspdy_dp_debug.so, compiled with SPDY_DEBUG_CHECKS), in which every row-buffer
+ * and table access of the forward kernels tests its index first and a bad access is recorded and skipped
+ * instead of performed: bit 1 = a read of the previous row (Algorithm 1's D[l-1, t - t_l^s]) outside the
+ * cells known to hold the row or +inf, bit 2 = a read that returned the marker of a cell not yet written,
+ * bit 3 = a store outside its row or table.  spdy_debug_checks_enabled() tells which build is loaded.
+ */
+int spdy_plan_status_word(spdy_plan *plan, void *cuda_stream, int32_t *word_host);
+int spdy_debug_checks_enabled(void);
 
 /*
  * Measurement aid.  With timing on, every spdy_solve_batch on this plan records CUDA events on

@@ -14,6 +14,10 @@ import numpy as np
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libspdy_dp.so")
+DEBUG_LIB_PATH = os.path.join(_PKG, "libspdy_dp_debug.so")  # same sources with index checks in the kernels
+HOST_LIB_PATH = os.path.join(_PKG, "libspdy_plan_host.so")  # spdy_plan.cpp alone: plans and host helpers
+
+SPDY_KERNEL_AUTO, SPDY_KERNEL_CTA, SPDY_KERNEL_WARP = 0, 1, 2
 
 SPDY_TABLE_DEFAULT, SPDY_TABLE_ARG_U8, SPDY_TABLE_ROW_F32 = 0, 1, 2
 
@@ -24,13 +28,32 @@ EXPORTS = (
     "spdy_solve_batch_static", "spdy_static_scratch_bytes", "spdy_strerror", "spdy_last_cuda_error", "spdy_version",
     "spdy_solve_batch_coeffs", "spdy_solve_batch_coeffs_host", "spdy_quadratic_errors",
     "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile", "spdy_probe_peaks",
+    "spdy_plan_get_tables", "spdy_plan_verify", "spdy_plan_status_word", "spdy_debug_checks_enabled",
+)
+# What the host-only library holds (everything that needs no CUDA).
+HOST_EXPORTS = (
+    "spdy_plan_create", "spdy_plan_destroy", "spdy_plan_get_info", "spdy_plan_get_bands", "spdy_workspace_bytes",
+    "spdy_plan_get_tables", "spdy_plan_verify", "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile",
+    "spdy_strerror", "spdy_version",
 )
 
 
 class SpdyOptions(ctypes.Structure):
     _fields_ = [("table_format", ctypes.c_int32), ("threads", ctypes.c_int32),
                 ("cluster", ctypes.c_int32), ("forward_mode", ctypes.c_int32),
-                ("rows_in_global", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3)]
+                ("rows_in_global", ctypes.c_int32), ("kernel", ctypes.c_int32),
+                ("schedule", ctypes.c_int32), ("auto_shape", ctypes.c_int32)]
+
+
+class SpdyPlanTables(ctypes.Structure):
+    _fields_ = [("L", ctypes.c_int32), ("K", ctypes.c_int32), ("kernel_kind", ctypes.c_int32),
+                ("threads", ctypes.c_int32), ("warps_per_candidate", ctypes.c_int32), ("cluster", ctypes.c_int32),
+                ("forward_mode", ctypes.c_int32), ("max_cells_per_lane", ctypes.c_int32),
+                ("row_stride", ctypes.c_int32), ("pad", ctypes.c_int32), ("out_stride", ctypes.c_int32),
+                ("win_stride", ctypes.c_int32), ("mask_words", ctypes.c_int32), ("n_passes", ctypes.c_int32),
+                ("pitch", ctypes.c_int64), ("layers", ctypes.c_void_p), ("slots", ctypes.c_void_p),
+                ("passes", ctypes.c_void_p), ("pass_masks", ctypes.c_void_p), ("pass_ptr", ctypes.c_void_p),
+                ("slices", ctypes.c_void_p)]
 
 
 class SpdyPlanInfo(ctypes.Structure):
@@ -43,7 +66,8 @@ class SpdyPlanInfo(ctypes.Structure):
                 ("band_cells", ctypes.c_int64), ("useful_updates", ctypes.c_int64),
                 ("issued_updates", ctypes.c_int64), ("nominal_updates", ctypes.c_int64),
                 ("distinct_updates", ctypes.c_int64), ("launches_per_wave", ctypes.c_int32),
-                ("reserved1", ctypes.c_int32)]
+                ("kernel", ctypes.c_int32), ("forward_mode", ctypes.c_int32), ("candidates_per_cta", ctypes.c_int32),
+                ("alternates", ctypes.c_int32), ("reserved1", ctypes.c_int32)]
 
     def as_dict(self) -> dict:
         return {name: int(getattr(self, name)) for name, _ in self._fields_}
@@ -54,22 +78,15 @@ class SpdyError(RuntimeError):
         self.status = status
         lib = _load()
         text = lib.spdy_strerror(status).decode()
-        extra = f" (cudaError {lib.spdy_last_cuda_error()})" if status == -4 else ""
+        extra = f" (cudaError {lib.spdy_last_cuda_error()})" if status == -4 and hasattr(lib, "spdy_last_cuda_error") else ""
         super().__init__(f"{where}: {text}{extra} [{status}]")
 
 
 _lib = None
+_loaded = {}
 
 
-def _load():
-    global _lib
-    if _lib is not None:
-        return _lib
-    if not os.path.exists(LIB_PATH):
-        raise RuntimeError(f"{LIB_PATH} is missing: build it with "
-                           "`python -m paper_2201_13096_b200.build` (needs nvcc); "
-                           "there is no fallback implementation")
-    lib = ctypes.CDLL(LIB_PATH)
+def _configure(lib, host_only: bool = False):
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
     lib.spdy_plan_create.restype = ctypes.c_int
     lib.spdy_plan_create.argtypes = [ctypes.POINTER(vp), vp, i32, i32, i32, ctypes.c_int,
@@ -80,8 +97,23 @@ def _load():
     lib.spdy_plan_get_info.argtypes = [vp, ctypes.POINTER(SpdyPlanInfo)]
     lib.spdy_plan_get_bands.restype = ctypes.c_int
     lib.spdy_plan_get_bands.argtypes = [vp, vp, vp]
+    lib.spdy_plan_get_tables.restype = ctypes.c_int
+    lib.spdy_plan_get_tables.argtypes = [vp, i32, ctypes.POINTER(SpdyPlanTables)]
+    lib.spdy_plan_verify.restype = ctypes.c_int
+    lib.spdy_plan_verify.argtypes = [vp]
     lib.spdy_workspace_bytes.restype = ctypes.c_size_t
     lib.spdy_workspace_bytes.argtypes = [vp, i64]
+    lib.spdy_time_target.restype = ctypes.c_double
+    lib.spdy_time_target.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double]
+    lib.spdy_bucketize_times.restype = ctypes.c_int
+    lib.spdy_bucketize_times.argtypes = [vp, i32, i32, ctypes.c_double, i32, i32, vp]
+    lib.spdy_uniform_profile.restype = ctypes.c_int
+    lib.spdy_uniform_profile.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i64)]
+    lib.spdy_strerror.restype = ctypes.c_char_p
+    lib.spdy_strerror.argtypes = [ctypes.c_int]
+    lib.spdy_version.restype = ctypes.c_int
+    if host_only:
+        return lib
     lib.spdy_solve_batch.restype = ctypes.c_int
     lib.spdy_solve_batch.argtypes = [vp, vp, i64, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.spdy_solve_batch_host.restype = ctypes.c_int
@@ -92,18 +124,15 @@ def _load():
     lib.spdy_solve_batch_coeffs_host.argtypes = [vp, vp, i64, vp, vp, vp, vp]
     lib.spdy_quadratic_errors.restype = ctypes.c_int
     lib.spdy_quadratic_errors.argtypes = [vp, i64, i32, i32, vp, vp]
-    lib.spdy_time_target.restype = ctypes.c_double
-    lib.spdy_time_target.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double]
-    lib.spdy_bucketize_times.restype = ctypes.c_int
-    lib.spdy_bucketize_times.argtypes = [vp, i32, i32, ctypes.c_double, i32, i32, vp]
-    lib.spdy_uniform_profile.restype = ctypes.c_int
-    lib.spdy_uniform_profile.argtypes = [vp, i32, i32, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i64)]
     lib.spdy_probe_peaks.restype = ctypes.c_int
     lib.spdy_probe_peaks.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     lib.spdy_solve_batch_simple.restype = ctypes.c_int
     lib.spdy_solve_batch_simple.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.spdy_plan_check_status.restype = ctypes.c_int
     lib.spdy_plan_check_status.argtypes = [vp, vp]
+    lib.spdy_plan_status_word.restype = ctypes.c_int
+    lib.spdy_plan_status_word.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    lib.spdy_debug_checks_enabled.restype = ctypes.c_int
     lib.spdy_plan_enable_timing.restype = ctypes.c_int
     lib.spdy_plan_enable_timing.argtypes = [vp, ctypes.c_int]
     lib.spdy_plan_last_timing.restype = ctypes.c_int
@@ -112,12 +141,37 @@ def _load():
     lib.spdy_solve_batch_static.restype = ctypes.c_int
     lib.spdy_solve_batch_static.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.spdy_static_scratch_bytes.restype = ctypes.c_size_t
-    lib.spdy_strerror.restype = ctypes.c_char_p
-    lib.spdy_strerror.argtypes = [ctypes.c_int]
     lib.spdy_last_cuda_error.restype = ctypes.c_int
-    lib.spdy_version.restype = ctypes.c_int
-    _lib = lib
     return lib
+
+
+def open_library(path: str, host_only: bool = False):
+    """Load and type one build of the library (cached per path); raises if the file is missing."""
+    if path not in _loaded:
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: build it with "
+                               "`python -m paper_2201_13096_b200.build` (needs nvcc); "
+                               "there is no fallback implementation")
+        _loaded[path] = _configure(ctypes.CDLL(path), host_only)
+    return _loaded[path]
+
+
+def select_library(which: str = "release"):
+    """Make every call of this module go to one build of the library: "release" (libspdy_dp.so, the
+    default), "debug" (libspdy_dp_debug.so, index checks inside the kernels) or "host"
+    (libspdy_plan_host.so: plans and host helpers only, no device).  Returns the library.  Plans made
+    with one build must not be handed to another."""
+    global _lib
+    path = {"release": LIB_PATH, "debug": DEBUG_LIB_PATH, "host": HOST_LIB_PATH}[which]
+    _lib = open_library(path, host_only=(which == "host"))
+    return _lib
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = open_library(LIB_PATH)
+    return _lib
 
 
 def library():
@@ -141,14 +195,17 @@ class Plan:
     """``spdy_plan``: everything that depends only on ``times`` and ``B``."""
 
     def __init__(self, times, B: int, device: int = 0, table_format: int = SPDY_TABLE_DEFAULT,
-                 threads: int = 0, cluster: int = 0, forward_mode: int = 0, rows_in_global: int = 0):
+                 threads: int = 0, cluster: int = 0, forward_mode: int = 0, rows_in_global: int = 0,
+                 kernel: int = SPDY_KERNEL_AUTO, schedule: int = 0, auto_shape: int = 0):
         lib = _load()
         t = np.ascontiguousarray(np.asarray(times), dtype=np.int32)
         if t.ndim != 2:
             raise ValueError("times must be [L][K]")
         self.L, self.K, self.B, self.device = int(t.shape[0]), int(t.shape[1]), int(B), int(device)
         opts = SpdyOptions(table_format=table_format, threads=threads, cluster=cluster,
-                           forward_mode=forward_mode, rows_in_global=rows_in_global)
+                           forward_mode=forward_mode, rows_in_global=rows_in_global, kernel=kernel,
+                           schedule=schedule, auto_shape=auto_shape)
+        self._lib = lib  # the build this plan belongs to
         handle = ctypes.c_void_p()
         _check(lib.spdy_plan_create(ctypes.byref(handle), t.ctypes.data_as(ctypes.c_void_p),
                                     self.L, self.K, self.B, self.device, ctypes.byref(opts)),
@@ -158,7 +215,7 @@ class Plan:
 
     def close(self):
         if getattr(self, "_h", None):
-            _load().spdy_plan_destroy(self._h)
+            self._lib.spdy_plan_destroy(self._h)
             self._h = None
         self._ws = None
 
@@ -180,6 +237,39 @@ class Plan:
 
     def workspace_bytes(self, N: int) -> int:
         return int(_load().spdy_workspace_bytes(self._h, int(N)))
+
+    def verify(self):
+        """``spdy_plan_verify``: the host-side proof that every access of the kernels stays in bounds."""
+        _check(_load().spdy_plan_verify(self._h), "spdy_plan_verify")
+
+    def tables(self, which: int = 0) -> dict:
+        """``spdy_plan_get_tables`` as NumPy copies: ``which`` 0 = main launch shape, -1 = the byte table's
+        merged set, i >= 1 = the i-th launch shape for small batches."""
+        t = SpdyPlanTables()
+        _check(_load().spdy_plan_get_tables(self._h, int(which), ctypes.byref(t)), "spdy_plan_get_tables")
+
+        def arr(ptr, ctype, shape):
+            n = int(np.prod(shape))
+            if not ptr or n == 0:
+                return np.zeros(shape, dtype=np.dtype(ctype))
+            return np.ctypeslib.as_array(ctypes.cast(ptr, ctypes.POINTER(ctype)), shape=(n,)).reshape(shape).copy()
+
+        out = {name: int(getattr(t, name)) for name, ct in SpdyPlanTables._fields_ if ct is not ctypes.c_void_p}
+        W = max(1, out["warps_per_candidate"])
+        out["layers"] = arr(t.layers, ctypes.c_int32, (out["L"], 8))
+        out["slots"] = arr(t.slots, ctypes.c_int32, (out["L"], out["K"], 2))
+        out["passes"] = arr(t.passes, ctypes.c_int32, (out["n_passes"], 2))
+        out["pass_masks"] = arr(t.pass_masks, ctypes.c_uint64, (out["n_passes"], out["mask_words"]))
+        out["pass_ptr"] = arr(t.pass_ptr, ctypes.c_int32, (out["L"] * W + 1,)) if t.pass_ptr else None
+        out["slices"] = arr(t.slices, ctypes.c_int32, (out["L"], out["cluster"], 8)) if t.slices else None
+        return out
+
+    def status_word(self, stream=None) -> int:
+        """``spdy_plan_status_word``: read and clear the self-check word (0 = nothing flagged)."""
+        word = ctypes.c_int32()
+        _check(_load().spdy_plan_status_word(self._h, _stream_handle(stream), ctypes.byref(word)),
+               "spdy_plan_status_word")
+        return int(word.value)
 
     def enable_timing(self, on: bool = True):
         _check(_load().spdy_plan_enable_timing(self._h, int(on)), "spdy_plan_enable_timing")

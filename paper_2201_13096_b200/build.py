@@ -1,21 +1,40 @@
-"""Compile the CUDA library in-tree for sm_100a with nvcc (cross-compiles without a GPU)."""
+"""Compile the library in-tree for sm_100a (nvcc cross-compiles without a GPU).
+
+Three shared objects come out of ``csrc/``:
+
+* ``libspdy_dp.so``        - the product: host plan (g++) + kernels and launch code (nvcc);
+* ``libspdy_dp_debug.so``  - the same sources with ``-DSPDY_DEBUG_CHECKS``: every row and table access of
+  the forward kernels checks its index and reports through the plan's status word (for tests);
+* ``libspdy_plan_host.so`` - ``spdy_plan.cpp`` alone, built with the host compiler: plans, their
+  verification and the host helpers, for machines and tests without nvcc.
+
+Translation units compile in parallel and only when they or a header changed.
+"""
 from __future__ import annotations
 
+import glob
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 PKG = os.path.dirname(os.path.abspath(__file__))
-SRC = os.path.join(PKG, "csrc", "spdy_dp.cu")
-HDR = os.path.join(os.path.dirname(PKG), "include", "spdy_dp.h")
+CSRC = os.path.join(PKG, "csrc")
+HEADERS = [os.path.join(os.path.dirname(PKG), "include", "spdy_dp.h"),
+           os.path.join(CSRC, "spdy_plan.h"), os.path.join(CSRC, "spdy_device.cuh")]
+HOST_SOURCE = os.path.join(CSRC, "spdy_plan.cpp")
 LIB = os.path.join(PKG, "libspdy_dp.so")
+LIB_DEBUG = os.path.join(PKG, "libspdy_dp_debug.so")
+LIB_HOST = os.path.join(PKG, "libspdy_plan_host.so")
+OBJ_ROOT = os.path.join(PKG, "_build")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-lineinfo", "-O3", "-std=c++17",
     "--fmad=false", "--ftz=false", "--prec-div=true", "--prec-sqrt=true",
-    "-shared", "-Xcompiler", "-fPIC",
+    "-Xcompiler", "-fPIC",
 ]
+GXX_FLAGS = ["-O2", "-std=c++17", "-fPIC", "-Wall", "-Wextra"]
 
 
 def _nvcc() -> str:
@@ -23,17 +42,75 @@ def _nvcc() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Build ``libspdy_dp.so`` next to this file unless it is newer than its sources."""
-    newest = max(os.path.getmtime(SRC), os.path.getmtime(HDR))
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest:
-        return LIB
-    tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [_nvcc(), *NVCC_FLAGS, *( ["-Xptxas", "-v"] if verbose else []), "-o", tmp, SRC]
-    subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+def cuda_sources() -> list:
+    return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
+
+
+def _newest(paths) -> float:
+    return max(os.path.getmtime(p) for p in paths)
+
+
+def _stale(target: str, deps) -> bool:
+    return (not os.path.exists(target)) or os.path.getmtime(target) < _newest(deps)
+
+
+def _run(cmd, log=None):
+    res = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+    if log is not None:
+        log.append(res.stdout)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout)
+        raise subprocess.CalledProcessError(res.returncode, cmd)
+
+
+def build_host(force: bool = False) -> str:
+    """``libspdy_plan_host.so``: the host side alone, host compiler only."""
+    if force or _stale(LIB_HOST, [HOST_SOURCE, HEADERS[0], HEADERS[1]]):
+        tmp = LIB_HOST + f".tmp{os.getpid()}"
+        _run(["g++", *GXX_FLAGS, "-shared", "-o", tmp, HOST_SOURCE])
+        os.replace(tmp, LIB_HOST)
+    return LIB_HOST
+
+
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Build ``libspdy_dp.so`` (or the debug library) next to this file unless it is newer than its
+    sources.  Returns the library's path; with ``verbose`` the compilers' output (``-Xptxas -v``) goes
+    to stdout."""
+    lib = LIB_DEBUG if debug else LIB
+    sources = cuda_sources()
+    if not force and not _stale(lib, sources + [HOST_SOURCE] + HEADERS):
+        return lib
+    objdir = os.path.join(OBJ_ROOT, "debug" if debug else "release")
+    os.makedirs(objdir, exist_ok=True)
+    defines = ["-DSPDY_DEBUG_CHECKS"] if debug else []
+    jobs, objects, log = [], [], []
+    for src in sources:
+        obj = os.path.join(objdir, os.path.basename(src) + ".o")
+        objects.append(obj)
+        if force or verbose or _stale(obj, [src] + HEADERS):
+            jobs.append([_nvcc(), *NVCC_FLAGS, *defines, *(["-Xptxas", "-v"] if verbose else []), "-c", "-o", obj, src])
+    host_obj = os.path.join(objdir, "spdy_plan.cpp.o")
+    objects.append(host_obj)
+    if force or _stale(host_obj, [HOST_SOURCE, HEADERS[0], HEADERS[1]]):
+        jobs.append(["g++", *GXX_FLAGS, *defines, "-c", "-o", host_obj, HOST_SOURCE])
+    with ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 1))) as pool:
+        list(pool.map(lambda cmd: _run(cmd, log), jobs))
+    tmp = lib + f".tmp{os.getpid()}"
+    _run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp, *objects])
+    os.replace(tmp, lib)
+    if verbose:
+        print("".join(log))
+    return lib
+
+
+def build_all(force: bool = False) -> None:
+    build(force=force)
+    build(force=force, debug=True)
+    build_host(force=force)
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--host" in sys.argv:
+        print(build_host(force="--force" in sys.argv))
+    else:
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -1,0 +1,930 @@
+// Device code of the batched SPDY dynamic program for B200 (sm_100a): the cell updates, the warp pass,
+// and the three forward kernels (one CTA, one thread-block cluster, or one warp per candidate).
+//
+// One candidate = one min-plus dynamic program over L layers (Section 3.2, Eq. 2-3) followed by the
+// final minimum over the budget axis; the walk back of Appendix A, Algorithm 1 runs in a second kernel.
+// The forward kernels keep two band-limited DP rows in shared memory (or, for very wide rows, in global
+// memory) and stream one table row per layer to global memory.
+//
+// Bit-exactness contract: every cell value is produced by exactly one fp32 round-to-nearest add
+// (previous-row value + error) and compared with strict "<" in ascending choice order, so the
+// results equal a plain sequential evaluation of Algorithm 1 with Eq. 2's bucket range.
+//
+// Built with -DSPDY_DEBUG_CHECKS every row-buffer and table access of the forward kernels tests its index
+// first: an access outside its buffer, or a read of a cell that holds neither the previous row nor +inf
+// (the new row's buffer is filled with NaN before each layer), sets a bit of the plan's status word and
+// is skipped - never a trap, never an early exit past a barrier.
+#ifndef SPDY_DEVICE_CUH
+#define SPDY_DEVICE_CUH
+
+#include "spdy_plan.h"
+
+#include <cooperative_groups.h>
+#include <cuda_runtime.h>
+
+namespace spdy {
+
+// Bits of the status word.
+constexpr int STATUS_WALK_BACK = 1;   // a table entry was not a valid choice, or the walk did not end at t = 0
+constexpr int STATUS_READ_RANGE = 2;  // debug build: a row read outside the region known to hold the row or +inf
+constexpr int STATUS_READ_STALE = 4;  // debug build: a row read returned the NaN that marks an unwritten cell
+constexpr int STATUS_WRITE_RANGE = 8; // debug build: a row or table store outside its buffer
+
+struct FwdArgs {
+    const float *errors;      // [N][L][K], or null when the errors follow from coefficients
+    const float *coeffs;      // [N][L] sensitivity coefficients (Eq. 4), used when errors is null
+    const float *qtab;        // [K]: fp32((i / (K - 1))^2)
+    const TapRange *slots;    // [L][K], the first layers[l].nslots of a layer are valid
+    const uint8_t *slot_ptr;     // [L][K+1]: members of slot u are slot_member[slot_ptr[u] .. slot_ptr[u+1])
+    const uint8_t *slot_member;  // [L][K]: choice indices grouped by slot
+    const LayerDesc *layers;  // [L]
+    const PassDesc *passes;   // warp passes grouped by (layer, warp)
+    const unsigned long long *pass_masks;  // per pass: one bit per slot that overlaps it
+    const int32_t *pass_ptr;  // [L * W + 1]
+    void *table;              // wave-local walk-back table
+    float *cost;              // [N]
+    int32_t *time_used;       // [N]
+    int32_t *status;          // the plan's status word
+    int64_t pitch;            // table cells per candidate
+    int64_t n_first;          // first candidate of this wave
+    int64_t n_count;          // candidates of this wave
+    int32_t L, K;
+    int32_t row_stride;       // floats per row buffer
+    int32_t pad;              // +inf guard cells on either side of a row
+    float *grows;             // row buffers in global memory (GROWS kernels), else null
+    int64_t grows_stride;     // floats between the row buffers of consecutive candidates
+    const uint8_t *cand_flags; // per candidate of the wave, or null: run only candidates whose flag == which
+    int32_t which;
+};
+
+struct ClusterArgs {
+    FwdArgs f;
+    const SliceDesc *slices;  // [L][C]
+    int32_t C;
+    int32_t out_stride;  // floats per `out` buffer
+    int32_t win_stride;  // floats of `win`
+};
+
+__device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
+
+// Error of choice k of layer l of candidate n: read from the table, or Eq. 4's c * (k / (K-1))^2 as
+// one fp32 multiply of the coefficient with the pre-rounded square.
+__device__ __forceinline__ float choice_error(const float *errors, const float *coeffs, const float *qtab,
+                                              const int64_t n, const int l, const int k, const int L, const int K)
+{
+    if (errors) return errors[(n * L + l) * K + k];
+    return __fmul_rn(coeffs[n * L + l], qtab[k]);
+}
+
+// (shift, error bits) of slot u of layer l for one candidate: the smallest error among the
+// slot's choices (a single choice unless equal times were merged).
+__device__ __forceinline__ int2 stage_slot(const FwdArgs &args, const int64_t n, const int l, const int u)
+{
+    const int K = args.K, L = args.L;
+    const uint8_t *ptr = args.slot_ptr + static_cast<size_t>(l) * (K + 1);
+    const uint8_t *member = args.slot_member + static_cast<size_t>(l) * K;
+    const int j0 = ptr[u], j1 = ptr[u + 1];
+    float e = choice_error(args.errors, args.coeffs, args.qtab, n, l, member[j0], L, K);
+    for (int j = j0 + 1; j < j1; ++j)
+        e = fminf(e, choice_error(args.errors, args.coeffs, args.qtab, n, l, member[j], L, K));
+    return make_int2(args.slots[static_cast<size_t>(l) * K + u].a, __float_as_int(e));
+}
+
+// What a pass may touch, for the debug build's index checks; empty otherwise.
+struct AccessWindow {
+#ifdef SPDY_DEBUG_CHECKS
+    int read_lo, read_hi;    // previous-row cells [read_lo, read_hi) hold the row or +inf
+    int write_hi;            // new-row cells [0, write_hi) may be stored
+    long long table_hi;      // table cells [0, table_hi) of this row may be stored
+    int32_t *status;
+#endif
+};
+
+// The previous row as one lane sees it through one slot: cell j of the lane is p[32 * j].
+struct Src {
+    const float *p;
+#ifdef SPDY_DEBUG_CHECKS
+    int cell;  // index of p[0] relative to band cell 0 of the previous row
+#endif
+    __device__ __forceinline__ float at(const int j, const AccessWindow &w) const
+    {
+#ifdef SPDY_DEBUG_CHECKS
+        const int c = cell + 32 * j;
+        if (c < w.read_lo || c >= w.read_hi) {
+            atomicOr(w.status, STATUS_READ_RANGE);
+            return pos_inf();
+        }
+        const float v = p[32 * j];
+        if (v != v) atomicOr(w.status, STATUS_READ_STALE);
+        return v;
+#else
+        (void)w;
+        return p[32 * j];
+#endif
+    }
+};
+
+__device__ __forceinline__ Src make_src(const float *prev, const int first_cell, const int shift)
+{
+    Src s;
+    s.p = prev + first_cell - shift;
+#ifdef SPDY_DEBUG_CHECKS
+    s.cell = first_cell - shift;
+#endif
+    return s;
+}
+
+// Two independent round-to-nearest fp32 adds in one instruction: (x, y) += (e, e).
+__device__ __forceinline__ void add2_rn(float &x, float &y, unsigned long long e2)
+{
+    unsigned long long p, r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "f"(x), "f"(y));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(p), "l"(e2));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(x), "=f"(y) : "l"(r));
+}
+
+__device__ __forceinline__ unsigned long long splat2(float e)
+{
+    unsigned long long p;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(p) : "f"(e));
+    return p;
+}
+
+__device__ __forceinline__ float min3(float a, float b, float c)
+{
+    float m;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+    return m;
+}
+
+// Cell updates of one slot (or two) on the RR cells a lane owns.
+template <int RR>
+__device__ __forceinline__ void update_min1(float (&best)[RR], const Src sa, const float ea, const AccessWindow &w)
+{
+#pragma unroll
+    for (int j = 0; j < RR; ++j) best[j] = fminf(best[j], __fadd_rn(sa.at(j, w), ea));
+}
+
+template <int RR>
+__device__ __forceinline__ void update_min2(float (&best)[RR], const Src sa, const float ea, const Src sb,
+                                            const float eb, const AccessWindow &w)
+{
+    const unsigned long long ea2 = splat2(ea), eb2 = splat2(eb);
+#pragma unroll
+    for (int j = 0; j + 1 < RR; j += 2) {
+        float a0 = sa.at(j, w), a1 = sa.at(j + 1, w);
+        float b0 = sb.at(j, w), b1 = sb.at(j + 1, w);
+        add2_rn(a0, a1, ea2);
+        add2_rn(b0, b1, eb2);
+        best[j] = min3(best[j], a0, b0);
+        best[j + 1] = min3(best[j + 1], a1, b1);
+    }
+    if (RR & 1) {
+        const float a0 = __fadd_rn(sa.at(RR - 1, w), ea);
+        const float b0 = __fadd_rn(sb.at(RR - 1, w), eb);
+        best[RR - 1] = min3(best[RR - 1], a0, b0);
+    }
+}
+
+template <int RR>
+__device__ __forceinline__ void update_arg(float (&best)[RR], int (&idx)[RR], const Src src, const float e,
+                                           const int k, const AccessWindow &w)
+{
+#pragma unroll
+    for (int j = 0; j < RR; ++j) {
+        const float v = __fadd_rn(src.at(j, w), e);
+        const bool better = v < best[j];  // strict: the lowest k keeps a tie
+        best[j] = better ? v : best[j];
+        idx[j] = better ? k : idx[j];
+    }
+}
+
+// Two slots k0 < k1 per step with the winning index read off the outcome: m = min(best, v0, v1); the cell
+// changes hands only if m < best (strict: a tie with the old value keeps the old, lower index), and then
+// to k0 if v0 attains m (a tie between the two goes to the lower index) and to k1 otherwise.  This is what
+// the scan "k0, then k1, strict <" leaves, at 2.5 instructions per update on top of load and add instead
+// of 3.  (A NaN sum never attains the minimum and never compares equal, as in the scan.)
+template <int RR>
+__device__ __forceinline__ void update_arg_pair(float (&best)[RR], int (&idx)[RR], const Src sa, const float ea,
+                                                const int k0, const Src sb, const float eb, const int k1,
+                                                const AccessWindow &w)
+{
+    const unsigned long long ea2 = splat2(ea), eb2 = splat2(eb);
+#define SPDY_PAIR_UPDATE(J, V0, V1)                     \
+    {                                                   \
+        const float m = min3(best[J], V0, V1);          \
+        const int kk = (V0 == m) ? k0 : k1;             \
+        idx[J] = (m < best[J]) ? kk : idx[J];           \
+        best[J] = m;                                    \
+    }
+#pragma unroll
+    for (int j = 0; j + 1 < RR; j += 2) {
+        float a0 = sa.at(j, w), a1 = sa.at(j + 1, w);
+        float b0 = sb.at(j, w), b1 = sb.at(j + 1, w);
+        add2_rn(a0, a1, ea2);
+        add2_rn(b0, b1, eb2);
+        SPDY_PAIR_UPDATE(j, a0, b0);
+        SPDY_PAIR_UPDATE(j + 1, a1, b1);
+    }
+    if (RR & 1) {
+        const float a0 = __fadd_rn(sa.at(RR - 1, w), ea);
+        const float b0 = __fadd_rn(sb.at(RR - 1, w), eb);
+        SPDY_PAIR_UPDATE(RR - 1, a0, b0);
+    }
+#undef SPDY_PAIR_UPDATE
+}
+
+// Same update as update_arg with the two selects written as predicated fp32 arithmetic that acts as an exact
+// move, to keep them off the integer/compare pipe: best <- v + (-0.0) (== v for every v) and
+// idx <- v * 0 + k (== k: a winning v is finite, so v * 0 is +-0).  The index is carried as a float.
+template <int RR>
+__device__ __forceinline__ void update_arg_pred(float (&best)[RR], float (&idxf)[RR], const Src src,
+                                                const float e, const int k, const AccessWindow &w)
+{
+    const float kf = static_cast<float>(k);
+    const unsigned long long e2 = splat2(e);
+#define SPDY_PRED_UPDATE(J, V)                        \
+    asm("{ .reg .pred p; setp.lt.f32 p, %2, %0;\n\t"  \
+        "@p add.rn.f32 %0, %2, 0f80000000;\n\t"       \
+        "@p fma.rn.f32 %1, %2, 0f00000000, %3; }"     \
+        : "+f"(best[J]), "+f"(idxf[J])                \
+        : "f"(V), "f"(kf))
+#pragma unroll
+    for (int j = 0; j + 1 < RR; j += 2) {
+        float v0 = src.at(j, w), v1 = src.at(j + 1, w);
+        add2_rn(v0, v1, e2);
+        SPDY_PRED_UPDATE(j, v0);
+        SPDY_PRED_UPDATE(j + 1, v1);
+    }
+    if (RR & 1) {
+        const float v0 = __fadd_rn(src.at(RR - 1, w), e);
+        SPDY_PRED_UPDATE(RR - 1, v0);
+    }
+#undef SPDY_PRED_UPDATE
+}
+
+// One warp pass: the 32*RR band cells starting at s (lane i owns cells s + i, s + i + 32, ...),
+// so every row access is lane-consecutive (conflict-free in shared memory) whatever the shift.  Both row
+// buffers carry guard cells of +inf on either side of the band: a pass that only partly overlaps a
+// slot's range reads +inf for the cells outside it and needs no per-cell bounds check (the host proves the
+// guard wide enough for every pass of a plan when the plan is built).  Which slots overlap the pass at all
+// is known on the host.  `krange` = u_lo | u_hi << 8 | dense << 16: the overlapping slots lie in
+// [u_lo, u_hi); when they are all of that range (dense, the usual case: times fall as the choice index
+// rises) the loop runs straight over it, otherwise it walks the set bits of `mask` (MW 64-bit words,
+// one bit per slot), in ascending order either way.
+//
+// `prev`/`cur` point at band cell 0 of the previous/new row; taps[u] = (a_u, bits of e_u): slot
+// u reads the previous row at t_rel - a_u.
+//
+// `prev` and `cur` carry no __restrict__: with the row buffers in global memory the kernel itself rewrites the
+// memory behind `prev` two layers later, so those reads must stay ordinary coherent loads.
+//
+// With MASKED only cells below `limit` are stored (a CTA of a cluster owns a slice of the band and
+// must not write its neighbour's cells); without it the caller guarantees room for the whole pass.
+template <int RR, int MODE, bool MASKED>
+__device__ __forceinline__ void process_span(const float *prev, float *cur, const int2 *__restrict__ taps,
+                                             const unsigned krange, const unsigned long long *__restrict__ mask,
+                                             const int MW, const int s, const int lane, void *table_row,
+                                             const int limit, const AccessWindow &w)
+{
+    const float INF = pos_inf();
+    const int first = s + lane;
+    const int k_lo = krange & 0xFF, k_hi = (krange >> 8) & 0xFF;
+    const bool dense = (krange >> 16) & 1;
+    float best[RR];
+#pragma unroll
+    for (int j = 0; j < RR; ++j) best[j] = INF;
+
+    auto store_allowed = [&](const int j) -> bool {
+        if (MASKED && !(s + j * 32 + lane < limit)) return false;
+#ifdef SPDY_DEBUG_CHECKS
+        if (s + j * 32 + lane >= w.write_hi || static_cast<long long>(s) + j * 32 + lane >= w.table_hi) {
+            atomicOr(w.status, STATUS_WRITE_RANGE);
+            return false;
+        }
+#endif
+        return true;
+    };
+
+    if constexpr (MODE == MODE_ROW2 || MODE == MODE_ROW) {
+        // Value-only minimum: the order of the slots does not matter, so overlapping slots
+        // are taken two at a time (MODE_ROW2) whatever their indices.
+        if (dense) {
+            int k = k_lo;
+            if (MODE == MODE_ROW2) {
+                // An odd first slot goes alone so that every pair below is one aligned 16-byte read.
+                if ((k & 1) && k < k_hi) {
+                    const int2 ta = taps[k];
+                    update_min1<RR>(best, make_src(prev, first, ta.x), __int_as_float(ta.y), w);
+                    ++k;
+                }
+#pragma unroll 1
+                for (; k + 1 < k_hi; k += 2) {
+                    const int4 t = *reinterpret_cast<const int4 *>(taps + k);
+                    update_min2<RR>(best, make_src(prev, first, t.x), __int_as_float(t.y), make_src(prev, first, t.z),
+                                    __int_as_float(t.w), w);
+                }
+            }
+#pragma unroll 1
+            for (; k < k_hi; ++k) {
+                const int2 ta = taps[k];
+                update_min1<RR>(best, make_src(prev, first, ta.x), __int_as_float(ta.y), w);
+            }
+        } else {
+#pragma unroll 1
+            for (int wd = 0; wd < MW; ++wd) {
+                unsigned long long m = __ldg(mask + wd);
+#pragma unroll 1
+                while (m) {
+                    const int2 ta = taps[64 * wd + __ffsll(static_cast<long long>(m)) - 1];
+                    m &= m - 1;
+                    update_min1<RR>(best, make_src(prev, first, ta.x), __int_as_float(ta.y), w);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < RR; ++j)
+            if (store_allowed(j)) cur[s + j * 32 + lane] = best[j];
+        float *D = static_cast<float *>(table_row) + s + lane;
+#pragma unroll
+        for (int j = 0; j < RR; ++j)
+            if (store_allowed(j)) D[j * 32] = best[j];
+    } else if constexpr (MODE == MODE_ARG || MODE == MODE_ARG_PAIR) {
+        int idx[RR];
+#pragma unroll
+        for (int j = 0; j < RR; ++j) idx[j] = 0xFF;
+        if (dense) {
+            int k = k_lo;
+            if (MODE == MODE_ARG_PAIR) {
+                if ((k & 1) && k < k_hi) {
+                    const int2 tp = taps[k];
+                    update_arg<RR>(best, idx, make_src(prev, first, tp.x), __int_as_float(tp.y), k, w);
+                    ++k;
+                }
+#pragma unroll 1
+                for (; k + 1 < k_hi; k += 2) {
+                    const int4 t = *reinterpret_cast<const int4 *>(taps + k);
+                    update_arg_pair<RR>(best, idx, make_src(prev, first, t.x), __int_as_float(t.y), k,
+                                        make_src(prev, first, t.z), __int_as_float(t.w), k + 1, w);
+                }
+            }
+#pragma unroll 1
+            for (; k < k_hi; ++k) {
+                const int2 tp = taps[k];
+                update_arg<RR>(best, idx, make_src(prev, first, tp.x), __int_as_float(tp.y), k, w);
+            }
+        } else {
+#pragma unroll 1
+            for (int wd = 0; wd < MW; ++wd) {
+                unsigned long long m = __ldg(mask + wd);
+#pragma unroll 1
+                while (m) {
+                    const int k = 64 * wd + __ffsll(static_cast<long long>(m)) - 1;
+                    m &= m - 1;
+                    const int2 tp = taps[k];
+                    update_arg<RR>(best, idx, make_src(prev, first, tp.x), __int_as_float(tp.y), k, w);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < RR; ++j)
+            if (store_allowed(j)) cur[s + j * 32 + lane] = best[j];
+        unsigned char *P = static_cast<unsigned char *>(table_row) + s + lane;
+#pragma unroll
+        for (int j = 0; j < RR; ++j)
+            if (store_allowed(j)) P[j * 32] = static_cast<unsigned char>(idx[j]);
+    } else {  // MODE_ARG_PRED
+        float idxf[RR];
+#pragma unroll
+        for (int j = 0; j < RR; ++j) idxf[j] = 255.0f;
+        if (dense) {
+#pragma unroll 1
+            for (int k = k_lo; k < k_hi; ++k) {
+                const int2 tp = taps[k];
+                update_arg_pred<RR>(best, idxf, make_src(prev, first, tp.x), __int_as_float(tp.y), k, w);
+            }
+        } else {
+#pragma unroll 1
+            for (int wd = 0; wd < MW; ++wd) {
+                unsigned long long m = __ldg(mask + wd);
+#pragma unroll 1
+                while (m) {
+                    const int k = 64 * wd + __ffsll(static_cast<long long>(m)) - 1;
+                    m &= m - 1;
+                    const int2 tp = taps[k];
+                    update_arg_pred<RR>(best, idxf, make_src(prev, first, tp.x), __int_as_float(tp.y), k, w);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < RR; ++j)
+            if (store_allowed(j)) cur[s + j * 32 + lane] = best[j];
+        unsigned char *P = static_cast<unsigned char *>(table_row) + s + lane;
+#pragma unroll
+        for (int j = 0; j < RR; ++j)
+            if (store_allowed(j)) P[j * 32] = static_cast<unsigned char>(static_cast<int>(idxf[j]));
+    }
+}
+
+// Runs the pass `pd` with the unrolled body for its cells-per-lane count (1..RCAP).
+template <int MODE, int RCAP, bool MASKED>
+__device__ __forceinline__ void run_pass(const int cpl, const float *prev, float *cur, const int2 *taps,
+                                         const unsigned krange, const unsigned long long *mask, const int MW,
+                                         const int s, const int lane, void *table_row, const int limit,
+                                         const AccessWindow &w)
+{
+    switch (cpl) {
+#define SPDY_CASE(RR)                                                                                          \
+    case RR:                                                                                                   \
+        if constexpr (RR <= kRmax && RR <= RCAP)                                                               \
+            process_span<RR, MODE, MASKED>(prev, cur, taps, krange, mask, MW, s, lane, table_row, limit, w);   \
+        break;
+        SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
+        SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
+        SPDY_CASE(13) SPDY_CASE(14) SPDY_CASE(15) SPDY_CASE(16) SPDY_CASE(17) SPDY_CASE(18)
+        SPDY_CASE(19) SPDY_CASE(20) SPDY_CASE(21) SPDY_CASE(22) SPDY_CASE(23) SPDY_CASE(24)
+#undef SPDY_CASE
+        default: break;
+    }
+}
+
+// (value, t) merge with the lowest t among equal values.
+__device__ __forceinline__ void warp_min_lowest_t(float &bv, int &bt)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+        const int ot = __shfl_xor_sync(0xffffffffu, bt, off);
+        if (ov < bv || (ov == bv && ot < bt)) {
+            bv = ov;
+            bt = ot;
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------------------------
+// One CTA per candidate
+// ----------------------------------------------------------------------------------------------
+//
+// RCAP: the largest cells-per-lane this instantiation can run.  The registers a kernel needs grow
+// with the largest unrolled pass, so plans whose passes are short use the RCAP = 8 build, which fits twice
+// as many CTAs per SM.
+//
+// GROWS: keep the two row buffers in global memory (args.grows) instead of shared memory.  This is the
+// fallback for bands too wide for one CTA's shared memory; the code is the same, the reads then go through
+// L1/L2.  Writes of one layer are ordered before the reads of the next by the same per-layer __syncthreads().
+//
+// The passes of a layer are laid out on the host per warp (pass_ptr): lengths chosen by the slots that
+// overlap them, dealt to the warps so that they arrive level at the one __syncthreads() per layer.
+template <int MODE, int NT, int MINB, int RCAP, bool GROWS>
+__global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs args)
+{
+    constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
+    constexpr int NWARPS = NT / 32;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *rows;
+    int2 *tap_buf;
+    if constexpr (GROWS) {
+        rows = args.grows + static_cast<size_t>(blockIdx.x) * static_cast<size_t>(args.grows_stride);
+        tap_buf = reinterpret_cast<int2 *>(smem_raw);
+    } else {
+        rows = reinterpret_cast<float *>(smem_raw);
+        tap_buf = reinterpret_cast<int2 *>(rows + 2 * static_cast<size_t>(args.row_stride));
+    }
+
+    // Two table sets may share a wave (see spdy_monotone_flags_kernel): a CTA whose candidate belongs
+    // to the other set leaves at once, before any barrier.
+    if (args.cand_flags && args.cand_flags[blockIdx.x] != args.which) return;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int L = args.L, K = args.K;
+    const int KS = (K + 1) & ~1;  // slots per staging buffer: even, so that slot pairs are 16-byte aligned
+    const int MW = (K + 63) >> 6;
+    const int64_t n_local = blockIdx.x;
+    const int64_t n = args.n_first + n_local;
+    const float INF = pos_inf();
+    const int PAD = args.pad;
+
+    // Both buffers start as +inf everywhere; D_0 is +0 at t = 0 (Eq. 3 via a virtual row 0).
+    LayerDesc ld = args.layers[0];
+    for (int i = tid; i < 2 * args.row_stride; i += NT) rows[i] = INF;
+    for (int u = tid; u < ld.nslots; u += NT) tap_buf[u] = stage_slot(args, n, 0, u);
+    int p0 = __ldg(args.pass_ptr + warp), p1 = __ldg(args.pass_ptr + warp + 1);
+    __syncthreads();
+    if (tid == 0) rows[PAD] = 0.0f;
+    __syncthreads();
+
+    for (int l = 0; l < L; ++l) {
+        const float *prev = rows + (l & 1) * args.row_stride + PAD;
+        float *cur = rows + ((l + 1) & 1) * args.row_stride + PAD;
+        const int2 *taps = tap_buf + (l & 1) * KS;
+
+        // Fetch the next layer's descriptor, pass range and slots early; the slots are parked in shared
+        // memory after the passes.  (NT >= K is guaranteed by the host, so one thread per slot suffices.)
+        LayerDesc ld_next = ld;
+        int q0 = 0, q1 = 0;
+        int2 next_tap = make_int2(0, 0);
+        bool have_next = false;
+        if (l + 1 < L) {
+            ld_next = args.layers[l + 1];
+            q0 = __ldg(args.pass_ptr + (l + 1) * NWARPS + warp);
+            q1 = __ldg(args.pass_ptr + (l + 1) * NWARPS + warp + 1);
+            have_next = tid < ld_next.nslots;
+            if (have_next) next_tap = stage_slot(args, n, l + 1, tid);
+        }
+
+        unsigned char *row_base = static_cast<unsigned char *>(args.table) +
+                                  (n_local * args.pitch + ld.rowoff) * (ROWFMT ? 4 : 1);
+        AccessWindow w;
+#ifdef SPDY_DEBUG_CHECKS
+        w.read_lo = -PAD;
+        w.read_hi = l == 0 ? args.row_stride - PAD : args.layers[l - 1].extent + PAD;
+        w.write_hi = ld.extent;
+        w.table_hi = args.pitch - ld.rowoff;
+        w.status = args.status;
+        for (int i = tid; i < ld.extent; i += NT) cur[i] = __int_as_float(0x7fc00000);  // mark the new row unwritten
+        __syncthreads();
+#endif
+        for (int p = p0; p < p1; ++p) {
+            const int2 pd = __ldg(reinterpret_cast<const int2 *>(args.passes + p));
+            run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+                                        args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
+        }
+        // Cells [width, extent) of the new row were written as +inf by the passes (they saw only +inf
+        // sources); PAD more cells of +inf behind them cover every read of the next layer.
+        for (int i = tid; i < PAD; i += NT) cur[ld.extent + i] = INF;
+        if (have_next) tap_buf[((l + 1) & 1) * KS + tid] = next_tap;
+        __syncthreads();
+        ld = ld_next;
+        p0 = q0;
+        p1 = q1;
+    }
+
+    // min over t <= B of D_L[t], lowest t among equals (the band's upper end never exceeds B).
+    const float *last = rows + (L & 1) * args.row_stride + PAD;
+    float bv = INF;
+    int bt = 0x7fffffff;
+    for (int t = tid; t < ld.width; t += NT) {
+        const float v = last[t];
+        if (v < bv) {
+            bv = v;
+            bt = t;
+        }
+    }
+    warp_min_lowest_t(bv, bt);
+    __shared__ float red_v[32];
+    __shared__ int red_t[32];
+    if (lane == 0) {
+        red_v[warp] = bv;
+        red_t[warp] = bt;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        bv = lane < NWARPS ? red_v[lane] : INF;
+        bt = lane < NWARPS ? red_t[lane] : 0x7fffffff;
+        warp_min_lowest_t(bv, bt);
+        if (lane == 0) {
+            const bool feasible = bv < INF;
+            args.cost[n] = feasible ? bv : INF;
+            args.time_used[n] = feasible ? ld.lo + bt : -1;
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------------------------
+// One warp per candidate
+// ----------------------------------------------------------------------------------------------
+//
+// For rows a pass or two wide (a budget of about a thousand buckets) a CTA per candidate spends more on
+// its per-layer barrier and fixed costs than on cell updates.  Here every warp of a CTA owns a candidate
+// outright: its own two row buffers and slot buffers in the CTA's shared memory, all passes of a layer, a
+// __syncwarp() where the CTA kernel has a __syncthreads().  Warps never wait for one another.  The host
+// offers this kernel only to plans whose layers have at most 64 shift slots (two staged per lane).
+constexpr int kWarpKernelThreads = 128;
+
+template <int MODE, int MINB, int RCAP>
+__global__ void __launch_bounds__(kWarpKernelThreads, MINB) spdy_forward_warp_kernel(const FwdArgs args)
+{
+    constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
+    constexpr int NWARPS = kWarpKernelThreads / 32;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int64_t n_local = static_cast<int64_t>(blockIdx.x) * NWARPS + warp;
+    if (n_local >= args.n_count) return;
+    if (args.cand_flags && args.cand_flags[n_local] != args.which) return;
+    const int L = args.L, K = args.K;
+    const int KS = (K + 1) & ~1;
+    const int MW = (K + 63) >> 6;
+    const int64_t n = args.n_first + n_local;
+    const float INF = pos_inf();
+    const int PAD = args.pad;
+    float *rows = reinterpret_cast<float *>(smem_raw) + static_cast<size_t>(warp) * 2 * args.row_stride;
+    int2 *tap_buf = reinterpret_cast<int2 *>(reinterpret_cast<float *>(smem_raw) + static_cast<size_t>(NWARPS) * 2 * args.row_stride) +
+                    static_cast<size_t>(warp) * 2 * KS;
+
+    LayerDesc ld = args.layers[0];
+    for (int i = lane; i < 2 * args.row_stride; i += 32) rows[i] = INF;
+    for (int u = lane; u < ld.nslots; u += 32) tap_buf[u] = stage_slot(args, n, 0, u);
+    int p0 = __ldg(args.pass_ptr), p1 = __ldg(args.pass_ptr + 1);
+    __syncwarp();
+    if (lane == 0) rows[PAD] = 0.0f;
+    __syncwarp();
+
+    for (int l = 0; l < L; ++l) {
+        const float *prev = rows + (l & 1) * args.row_stride + PAD;
+        float *cur = rows + ((l + 1) & 1) * args.row_stride + PAD;
+        const int2 *taps = tap_buf + (l & 1) * KS;
+
+        LayerDesc ld_next = ld;
+        int q0 = 0, q1 = 0;
+        int2 next_a = make_int2(0, 0), next_b = make_int2(0, 0);
+        if (l + 1 < L) {
+            ld_next = args.layers[l + 1];
+            q0 = __ldg(args.pass_ptr + l + 1);
+            q1 = __ldg(args.pass_ptr + l + 2);
+            if (lane < ld_next.nslots) next_a = stage_slot(args, n, l + 1, lane);
+            if (lane + 32 < ld_next.nslots) next_b = stage_slot(args, n, l + 1, lane + 32);
+        }
+
+        unsigned char *row_base = static_cast<unsigned char *>(args.table) +
+                                  (n_local * args.pitch + ld.rowoff) * (ROWFMT ? 4 : 1);
+        AccessWindow w;
+#ifdef SPDY_DEBUG_CHECKS
+        w.read_lo = -PAD;
+        w.read_hi = l == 0 ? args.row_stride - PAD : args.layers[l - 1].extent + PAD;
+        w.write_hi = ld.extent;
+        w.table_hi = args.pitch - ld.rowoff;
+        w.status = args.status;
+        for (int i = lane; i < ld.extent; i += 32) cur[i] = __int_as_float(0x7fc00000);
+        __syncwarp();
+#endif
+        for (int p = p0; p < p1; ++p) {
+            const int2 pd = __ldg(reinterpret_cast<const int2 *>(args.passes + p));
+            run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+                                        args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
+        }
+        for (int i = lane; i < PAD; i += 32) cur[ld.extent + i] = INF;
+        if (l + 1 < L) {
+            if (lane < ld_next.nslots) tap_buf[((l + 1) & 1) * KS + lane] = next_a;
+            if (lane + 32 < ld_next.nslots) tap_buf[((l + 1) & 1) * KS + lane + 32] = next_b;
+        }
+        __syncwarp();
+        ld = ld_next;
+        p0 = q0;
+        p1 = q1;
+    }
+
+    const float *last = rows + (L & 1) * args.row_stride + PAD;
+    float bv = INF;
+    int bt = 0x7fffffff;
+    for (int t = lane; t < ld.width; t += 32) {
+        const float v = last[t];
+        if (v < bv) {
+            bv = v;
+            bt = t;
+        }
+    }
+    warp_min_lowest_t(bv, bt);
+    if (lane == 0) {
+        const bool feasible = bv < INF;
+        args.cost[n] = feasible ? bv : INF;
+        args.time_used[n] = feasible ? ld.lo + bt : -1;
+    }
+}
+
+// ----------------------------------------------------------------------------------------------
+// One candidate per thread-block cluster
+// ----------------------------------------------------------------------------------------------
+//
+// For batches with fewer candidates than SMs (or on request) the band of every row is cut into C
+// contiguous slices, one per CTA of a cluster.  Each CTA keeps its slice of the new row in its own shared
+// memory (`out`, double buffered) and, before a layer, gathers the window of the previous row its slice
+// depends on - its own slice plus up to max_k a_k cells to the left - from the `out` buffers of its cluster
+// peers through distributed shared memory into a private window (`win`).  The cell updates then
+// run on local shared memory exactly as in the single-CTA kernel.  One hardware cluster barrier
+// per layer orders "slices of row l written" before "windows for row l+1 gathered"; every thread
+// of every CTA reaches every barrier (there is no early exit), so the barrier cannot wait forever.
+template <int MODE, int NT>
+__global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const ClusterArgs cargs)
+{
+    namespace cg = cooperative_groups;
+    constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
+    constexpr int NWARPS = NT / 32;
+    const FwdArgs &args = cargs.f;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int C = cargs.C;
+    const int rank = static_cast<int>(cluster.block_rank());
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *out = reinterpret_cast<float *>(smem_raw);                 // [2][out_stride]
+    float *win = out + 2 * static_cast<size_t>(cargs.out_stride);     // [win_stride]
+    int2 *tap_buf = reinterpret_cast<int2 *>(win + cargs.win_stride);  // [2][K]
+    __shared__ float cl_v[16];
+    __shared__ int cl_t[16];
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int L = args.L, K = args.K;
+    const int KS = (K + 1) & ~1;
+    const int64_t n_local = blockIdx.x / C;
+    const int64_t n = args.n_first + n_local;
+    const float INF = pos_inf();
+
+    // Virtual row 0: +0 at t = 0, held in rank 0's first `out` buffer.
+    for (int i = tid; i < 2 * cargs.out_stride; i += NT) out[i] = INF;
+    for (int u = tid; u < args.layers[0].nslots; u += NT) tap_buf[u] = stage_slot(args, n, 0, u);
+    __syncthreads();
+    if (rank == 0 && tid == 0) out[0] = 0.0f;
+    cluster.sync();
+
+    int prev_width = 1;
+    for (int l = 0; l < L; ++l) {
+        const SliceDesc sd = cargs.slices[l * C + rank];
+        const LayerDesc ld = args.layers[l];
+        const int2 *taps = tap_buf + (l & 1) * KS;
+        float *out_prev = out + (l & 1) * cargs.out_stride;
+        float *out_cur = out + ((l + 1) & 1) * cargs.out_stride;
+
+        int2 next_tap = make_int2(0, 0);
+        const bool have_next = (l + 1 < L) && (tid < args.layers[l + 1].nslots);
+        if (have_next) next_tap = stage_slot(args, n, l + 1, tid);
+
+        // Gather the window [q0, q0 + win_len) of the previous row, peer by peer; cells outside
+        // the previous band read as +inf.
+        {
+            const int q_end = sd.q0 + sd.win_len;
+            for (int i = tid; i < sd.win_len; i += NT) {
+                const int q = sd.q0 + i;
+                if (q < 0 || q >= prev_width) win[i] = INF;
+            }
+            const int q_lo = max(sd.q0, 0), q_hi = min(q_end, prev_width);
+            if (q_hi > q_lo) {
+                const int first_rank = q_lo / sd.prev_slice;
+                const int last_rank = (q_hi - 1) / sd.prev_slice;
+                for (int src = first_rank; src <= last_rank; ++src) {
+                    const int seg_lo = max(q_lo, src * sd.prev_slice);
+                    const int seg_hi = min(q_hi, (src + 1) * sd.prev_slice);
+                    const float *remote = (src == rank) ? out_prev : cluster.map_shared_rank(out_prev, src);
+                    const float *from = remote + (seg_lo - src * sd.prev_slice);
+                    float *to = win + (seg_lo - sd.q0);
+#ifdef SPDY_DEBUG_CHECKS
+                    if (src < 0 || src >= C || seg_lo - src * sd.prev_slice < 0 ||
+                        seg_hi - src * sd.prev_slice > cargs.out_stride || seg_hi - sd.q0 > cargs.win_stride) {
+                        if (tid == 0) atomicOr(args.status, STATUS_READ_RANGE);
+                        continue;
+                    }
+#endif
+                    for (int i = tid; i < seg_hi - seg_lo; i += NT) to[i] = from[i];
+                }
+            }
+        }
+        __syncthreads();
+
+        const float *prev = win - sd.q0;          // prev[q] for q in [q0, q0 + win_len)
+        float *cur = out_cur - sd.slice_lo;       // cur[t_rel] for t_rel in the slice
+        unsigned char *row_base = static_cast<unsigned char *>(args.table) +
+                                  (n_local * args.pitch + ld.rowoff) * (ROWFMT ? 4 : 1);
+        const int MW = (K + 63) >> 6;
+        AccessWindow w;
+#ifdef SPDY_DEBUG_CHECKS
+        w.read_lo = sd.q0;
+        w.read_hi = sd.q0 + sd.win_len;
+        w.write_hi = sd.slice_hi;
+        w.table_hi = args.pitch - ld.rowoff;
+        w.status = args.status;
+#endif
+        // All passes of a slice have one length: pick the unrolled body once, outside the pass loop.
+        switch (sd.cpl) {
+#define SPDY_CASE(RR)                                                                                             \
+    case RR:                                                                                                      \
+        if constexpr (RR <= kRmax)                                                                                \
+            for (int span = warp; span < sd.nspans; span += NWARPS) {                                             \
+                const int p = sd.mask_off + span;                                                                 \
+                const int2 pd = __ldg(reinterpret_cast<const int2 *>(args.passes + p));                           \
+                process_span<RR, MODE, true>(prev, cur, taps, static_cast<unsigned>(pd.y),                        \
+                                             args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane,       \
+                                             row_base, sd.slice_hi, w);                                           \
+            }                                                                                                     \
+        break;
+            SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
+            SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
+            SPDY_CASE(13) SPDY_CASE(14) SPDY_CASE(15) SPDY_CASE(16) SPDY_CASE(17) SPDY_CASE(18)
+            SPDY_CASE(19) SPDY_CASE(20) SPDY_CASE(21) SPDY_CASE(22) SPDY_CASE(23) SPDY_CASE(24)
+#undef SPDY_CASE
+            default: break;
+        }
+        if (have_next) tap_buf[((l + 1) & 1) * KS + tid] = next_tap;
+        prev_width = ld.width;
+        cluster.sync();  // slices of row l+1 complete everywhere; row l no longer needed
+    }
+
+    // Local minimum over the slice of the last row, then across the cluster through rank 0.
+    const SliceDesc sd = cargs.slices[(L - 1) * C + rank];
+    const LayerDesc ld = args.layers[L - 1];
+    const float *last = out + (L & 1) * cargs.out_stride;
+    float bv = INF;
+    int bt = 0x7fffffff;
+    for (int t = sd.slice_lo + tid; t < sd.slice_hi; t += NT) {
+        const float v = last[t - sd.slice_lo];
+        if (v < bv) {
+            bv = v;
+            bt = t;
+        }
+    }
+    warp_min_lowest_t(bv, bt);
+    __shared__ float red_v[32];
+    __shared__ int red_t[32];
+    if (lane == 0) {
+        red_v[warp] = bv;
+        red_t[warp] = bt;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        bv = lane < NWARPS ? red_v[lane] : INF;
+        bt = lane < NWARPS ? red_t[lane] : 0x7fffffff;
+        warp_min_lowest_t(bv, bt);
+        if (lane == 0) {
+            float *dst_v = cluster.map_shared_rank(cl_v, 0);
+            int *dst_t = cluster.map_shared_rank(cl_t, 0);
+            dst_v[rank] = bv;
+            dst_t[rank] = bt;
+        }
+    }
+    cluster.sync();
+    if (rank == 0 && tid == 0) {
+        bv = cl_v[0];
+        bt = cl_t[0];
+        for (int r = 1; r < C; ++r) {
+            if (cl_v[r] < bv || (cl_v[r] == bv && cl_t[r] < bt)) {
+                bv = cl_v[r];
+                bt = cl_t[r];
+            }
+        }
+        const bool feasible = bv < INF;
+        args.cost[n] = feasible ? bv : INF;
+        args.time_used[n] = feasible ? ld.lo + bt : -1;
+    }
+}
+
+// ----------------------------------------------------------------------------------------------
+// Kernel tables: each forward mode is compiled in a translation unit of its own
+// ----------------------------------------------------------------------------------------------
+
+using FwdKernel = void (*)(const FwdArgs);
+using ClusterKernel = void (*)(const ClusterArgs);
+
+struct FwdVariant {
+    int kind;     // KernelKind
+    int mode;
+    int threads;
+    int rcap;
+    FwdKernel fn;
+};
+
+struct ClusterVariant {
+    int mode;
+    int threads;
+    ClusterKernel fn;
+};
+
+struct VariantList {
+    const FwdVariant *fwd;
+    int n_fwd;
+    const ClusterVariant *cluster;
+    int n_cluster;
+};
+
+VariantList variants_arg();
+VariantList variants_arg_pred();
+VariantList variants_arg_pair();
+VariantList variants_row();
+VariantList variants_row2();
+
+// The standard set of builds of one mode.  FULL adds the rows-in-global build and the warp-per-candidate
+// builds, which only the default cell update of each table format has.
+#define SPDY_CTA_VARIANT(MODE, NT, MINB, RCAP) \
+    FwdVariant { KERNEL_CTA, MODE, NT, RCAP, spdy_forward_kernel<MODE, NT, MINB, RCAP, false> }
+// A 256-thread CTA of the pairwise argmin update (two register arrays of cells per lane) needs more than the
+// 80 registers that three resident CTAs leave: it runs two per SM.  cells_per_lane_1024() is the longest pass
+// a 1024-thread CTA (64 registers per thread) can unroll without spilling.
+template <int MODE> constexpr int ctas_256() { return MODE == MODE_ARG_PAIR ? 2 : 3; }
+#define SPDY_CTA_VARIANTS(MODE)                                                                                 \
+    SPDY_CTA_VARIANT(MODE, 128, 4, kRmax), SPDY_CTA_VARIANT(MODE, 256, ctas_256<MODE>(), kRmax),                  \
+    SPDY_CTA_VARIANT(MODE, 512, 1, kRmax), SPDY_CTA_VARIANT(MODE, 1024, 1, cells_per_lane_1024(MODE)),          \
+    SPDY_CTA_VARIANT(MODE, 128, 6, 8), SPDY_CTA_VARIANT(MODE, 256, 3, 8),                                       \
+    SPDY_CTA_VARIANT(MODE, 512, 1, 8), SPDY_CTA_VARIANT(MODE, 1024, 1, 8)
+#define SPDY_FULL_VARIANTS(MODE)                                                                                \
+    SPDY_CTA_VARIANTS(MODE),                                                                                    \
+    FwdVariant{KERNEL_CTA_GLOBAL, MODE, 1024, 12, spdy_forward_kernel<MODE, 1024, 1, 12, true>},                \
+    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, 8, spdy_forward_warp_kernel<MODE, 8, 8>},                 \
+    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, 16, spdy_forward_warp_kernel<MODE, 5, 16>},               \
+    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, kRmax, spdy_forward_warp_kernel<MODE, 4, kRmax>}
+#define SPDY_CLUSTER_VARIANTS(MODE) \
+    ClusterVariant{MODE, 256, spdy_forward_cluster_kernel<MODE, 256>}, ClusterVariant{MODE, 512, spdy_forward_cluster_kernel<MODE, 512>}
+
+}  // namespace spdy
+
+#endif  // SPDY_DEVICE_CUH

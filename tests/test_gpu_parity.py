@@ -140,10 +140,10 @@ def test_small_workspace_runs_in_waves(fmt):
 
 
 @pytest.mark.parametrize("threads", [128, 256, 512, 1024])
-@pytest.mark.parametrize("mode", [1, 2, 3, 4])
+@pytest.mark.parametrize("mode", [1, 2, 3, 4, 5])
 def test_every_launch_shape_and_cell_update_variant_gives_the_same_answer(threads, mode):
     wl = W.make_workload(2, N=8)
-    fmt = 1 if mode in (1, 2) else 2
+    fmt = 1 if mode in (1, 2, 5) else 2
     ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
     assert_same(gpu_solve(wl, fmt, threads=threads, forward_mode=mode), ref)
     tiny = W.tiny_random_instance(10_007, exact=True, N=5)
@@ -254,11 +254,12 @@ def test_sweep_points_with_few_candidates_every_candidate():
 
 
 @pytest.mark.parametrize("cluster", [2, 4, 8])
-@pytest.mark.parametrize("mode", [1, 2, 3, 4])
+@pytest.mark.parametrize("mode", [1, 3, 4, 5])
 def test_cluster_split_of_one_candidate_gives_the_same_answer(cluster, mode):
     """A candidate cut over a thread-block cluster (slices of every row, windows gathered through
-    distributed shared memory) must match the oracle like the single-CTA kernel."""
-    fmt = 1 if mode in (1, 2) else 2
+    distributed shared memory) must match the oracle like the single-CTA kernel.  (The predicated-move
+    update, mode 2, has no cluster build.)"""
+    fmt = 1 if mode in (1, 5) else 2
     wl = W.make_workload(2, N=6)
     ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
     assert_same(gpu_solve(wl, fmt, cluster=cluster, forward_mode=mode), ref)
@@ -534,10 +535,16 @@ def test_random_shapes_formats_and_launch_options():
         wl = W.Workload(f"fuzz-{trial}", times, errors, B)
         ref = oracle.solve_batch(wl.errors, wl.times, wl.B)
         options = [dict(), dict(cluster=int(rng.choice([2, 4, 8]))), dict(rows_in_global=1),
-                   dict(threads=int(rng.choice([256, 512, 1024])))]
+                   dict(threads=int(rng.choice([256, 512, 1024]))), dict(kernel=binding.SPDY_KERNEL_WARP),
+                   dict(kernel=binding.SPDY_KERNEL_CTA, schedule=1), dict(schedule=int(rng.integers(1, 9)) << 8)]
         for fmt in FORMATS:
             kw = options[int(rng.integers(len(options)))]
-            assert_same(gpu_solve(wl, fmt, **kw), ref), (trial, fmt, kw)
+            try:
+                got = gpu_solve(wl, fmt, **kw)
+            except binding.SpdyError as e:  # a warp per candidate stages at most 64 shift slots per layer
+                assert e.status == -3 and kw.get("kernel") == binding.SPDY_KERNEL_WARP, (trial, fmt, kw)
+                continue
+            assert_same(got, ref), (trial, fmt, kw)
 
 
 @pytest.mark.parametrize("fmt", FORMATS)
@@ -547,7 +554,7 @@ def test_two_live_plans_of_one_kernel_variant(fmt):
     point: the shared-memory limit is a property of the kernel on the device, not of a plan."""
     import torch
 
-    wide = W.make_workload(2, N=12)
+    wide = W.make_workload(1, N=12)
     narrow = W.make_workload(4, N=12, B=2500)
     ref_wide = oracle.solve_batch(wide.errors, wide.times, wide.B, threads=CORES)
     ref_narrow = oracle.solve_batch(narrow.errors, narrow.times, narrow.B, threads=CORES)
@@ -579,3 +586,81 @@ def test_plan_level_infeasible_budget_fills_every_candidate():
     torch.cuda.synchronize()
     assert (p == 0xFF).all().item() and (t == -1).all().item() and torch.isposinf(c).all().item()
     plan.close()
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_one_warp_per_candidate_gives_the_same_answer(fmt):
+    """The kernel for narrow rows (a warp owns a candidate; four candidates per CTA, no block barrier): chosen
+    by itself at B = 1000, forced on wider and on tiny shapes, batch sizes that leave warps of the last CTA idle."""
+    import torch
+
+    wl = W.make_workload(4, N=203, B=1000)
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+    assert plan.info["kernel"] == binding.SPDY_KERNEL_WARP and plan.info["candidates_per_cta"] == 4
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+    for n in (203, 1, 2, 5):
+        p, c, t = binding.solve_batch(plan, torch.from_numpy(wl.errors[:n]).cuda())
+        torch.cuda.synchronize()
+        plan.check_status()
+        assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), tuple(x[:n] for x in ref))
+    ws = torch.empty(plan.workspace_bytes(10), dtype=torch.uint8, device="cuda")  # waves of 10 candidates
+    p, c, t = binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda(), workspace=ws)
+    torch.cuda.synchronize()
+    assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), ref)
+    assert_same(binding.solve_batch_host(plan, wl.errors), ref)
+    plan.close()
+    for cfg, B, n in ((4, 2500, 9), (1, None, 5), (2, None, 5)):  # several passes per layer in one warp
+        wide = W.make_workload(cfg, N=n, B=B)
+        assert_same(gpu_solve(wide, fmt, kernel=binding.SPDY_KERNEL_WARP),
+                    oracle.solve_batch(wide.errors, wide.times, wide.B, threads=CORES))
+    for seed in range(60):
+        for exact in (False, True):
+            tiny = W.tiny_random_instance(seed + (10_000 if exact else 0), exact=exact, N=6)
+            assert_same(gpu_solve(tiny, fmt, kernel=binding.SPDY_KERNEL_WARP),
+                        oracle.solve_batch(tiny.errors, tiny.times, tiny.B))
+    wl2 = W.make_workload(2, N=1)
+    c = np.random.default_rng(3).uniform(0, 1, size=(37, wl.L)).astype(np.float32)
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+    p, cost, t = binding.solve_batch_coeffs(plan, torch.from_numpy(c).cuda())
+    torch.cuda.synchronize()
+    assert_same((p.cpu().numpy(), cost.cpu().numpy(), t.cpu().numpy()),
+                oracle.solve_batch(oracle.quadratic_errors(c, wl.K), wl.times, wl.B, threads=CORES))
+    plan.close()
+    del wl2
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_pass_schedules_give_the_same_answer(fmt):
+    """Passes sized by cost (default), passes of one size dealt round-robin, and capped pass lengths."""
+    wl = W.make_workload(2, N=6)
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+    for schedule in (0, 1, 5 << 8, 1 | (3 << 8), 16 << 8):
+        for threads in (128, 512):
+            assert_same(gpu_solve(wl, fmt, schedule=schedule, threads=threads), ref)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_small_batches_pick_their_launch_shape_by_themselves(fmt):
+    """With the launch shape left open, batches that cannot fill the device run as clusters or larger CTAs;
+    the answer does not depend on it, nor on the workspace being too small for that choice."""
+    import torch
+
+    wl = W.make_workload(2, N=300)
+    ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
+    plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+    assert plan.info["alternates"] >= 4
+    errors = torch.from_numpy(wl.errors).cuda()
+    for n in (1, 3, 18, 19, 37, 38, 74, 75, 148, 149, 295, 296, 300):
+        p, c, t = binding.solve_batch(plan, errors[:n])
+        torch.cuda.synchronize()
+        plan.check_status()
+        assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), tuple(x[:n] for x in ref))
+    pinned = binding.Plan(wl.times, wl.B, device=0, table_format=fmt, auto_shape=1)
+    tight = torch.empty(pinned.workspace_bytes(2), dtype=torch.uint8, device="cuda")
+    p, c, t = binding.solve_batch(plan, errors[:7], workspace=tight)  # waves of the main shape
+    torch.cuda.synchronize()
+    assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), tuple(x[:7] for x in ref))
+    assert_same(binding.solve_batch_host(plan, wl.errors[:20]), tuple(x[:20] for x in ref))
+    assert_same(binding.solve_batch_host(plan, wl.errors[:160]), tuple(x[:160] for x in ref))
+    plan.close()
+    pinned.close()
