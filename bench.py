@@ -79,6 +79,9 @@ def parse_args():
     ap.add_argument("--mode", type=int, default=0, help="forward kernel variant (see spdy_options.forward_mode)")
     ap.add_argument("--cluster", type=int, default=0, help="CTAs per candidate (0 = plan's choice)")
     ap.add_argument("--rows-in-global", type=int, default=0, help="1: row buffers in the workspace (wide-band fallback)")
+    ap.add_argument("--kernel", type=int, default=0, help="1: one CTA per candidate, 2: one warp per candidate (0 = plan's choice)")
+    ap.add_argument("--schedule", type=int, default=0, help="pass schedule (see spdy_options.schedule)")
+    ap.add_argument("--auto-shape", type=int, default=0, help="1: never switch launch shape for small batches")
     ap.add_argument("--search", type=int, default=0, metavar="TRIALS",
                     help="also run Algorithm 4 with this many trials per loop on the workload's timing table "
                          "(synthetic loss) and report where the time goes, under the key 'search'")
@@ -265,9 +268,10 @@ def run_ours(args):
     assert np.array_equal(probe.times, wl.times)
     fmt = {"default": 0, "arg": 1, "row": 2}[args.table]
     if args.mode:
-        fmt = 1 if args.mode in (1, 2) else 2
+        fmt = 1 if args.mode in (1, 2, 5) else 2
     plan = binding.Plan(wl.times, wl.B, device=local_rank, table_format=fmt, threads=args.threads,
-                        forward_mode=args.mode, cluster=args.cluster, rows_in_global=args.rows_in_global)
+                        forward_mode=args.mode, cluster=args.cluster, rows_in_global=args.rows_in_global,
+                        kernel=args.kernel, schedule=args.schedule, auto_shape=args.auto_shape)
     info = plan.info
     plan.enable_timing(True)
 

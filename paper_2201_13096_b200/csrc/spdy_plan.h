@@ -128,7 +128,7 @@ struct spdy_plan {
     int cluster = 1;
     int table_format = SPDY_TABLE_ROW_F32;
     int ctas_per_sm = 0;
-    int schedule = 0;        // 0 = cost-balanced passes, 1 = uniform passes dealt round-robin
+    int schedule = 0;        // 0 = passes of one length dealt round-robin, 1 = cost-sized passes dealt by load
     int pass_cap = 0;        // upper limit of cells per lane per pass asked for by the options (0 = the kernel's)
     spdy::DeviceLimits limits;
     int64_t smem_bytes = 0;

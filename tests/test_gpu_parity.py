@@ -631,7 +631,7 @@ def test_one_warp_per_candidate_gives_the_same_answer(fmt):
 
 @pytest.mark.parametrize("fmt", FORMATS)
 def test_pass_schedules_give_the_same_answer(fmt):
-    """Passes sized by cost (default), passes of one size dealt round-robin, and capped pass lengths."""
+    """Passes of one size dealt round-robin (default), passes sized by cost, and capped pass lengths."""
     wl = W.make_workload(2, N=6)
     ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
     for schedule in (0, 1, 5 << 8, 1 | (3 << 8), 16 << 8):
