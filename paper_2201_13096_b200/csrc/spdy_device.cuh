@@ -203,7 +203,9 @@ __device__ __forceinline__ void update_arg(float (&best)[RR], int (&idx)[RR], co
 // changes hands only if m < best (strict: a tie with the old value keeps the old, lower index), and then
 // to k0 if v0 attains m (a tie between the two goes to the lower index) and to k1 otherwise.  This is what
 // the scan "k0, then k1, strict <" leaves, at 2.5 instructions per update on top of load and add instead
-// of 3.  (A NaN sum never attains the minimum and never compares equal, as in the scan.)
+// of 3.  (A NaN sum never attains the minimum and never compares equal, as in the scan.)  A form that keeps
+// the index as a float and moves it under a predicate on the fp32 pipe (set, subtract, compare, predicated
+// add) has the same instruction count, loads the compare pipe less and measured 5 % slower.
 template <int RR>
 __device__ __forceinline__ void update_arg_pair(float (&best)[RR], int (&idx)[RR], const Src sa, const float ea,
                                                 const int k0, const Src sb, const float eb, const int k1,
@@ -356,6 +358,7 @@ __device__ __forceinline__ void process_span(const float *prev, float *cur, cons
         if (dense) {
             int k = k_lo;
             if (MODE == MODE_ARG_PAIR) {
+                // An odd first slot goes alone so that every pair below is one aligned 16-byte read.
                 if ((k & 1) && k < k_hi) {
                     const int2 tp = taps[k];
                     update_arg<RR>(best, idx, make_src(prev, first, tp.x), __int_as_float(tp.y), k, w);
@@ -546,8 +549,11 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         for (int i = tid; i < ld.extent; i += NT) cur[i] = __int_as_float(0x7fc00000);  // mark the new row unwritten
         __syncthreads();
 #endif
+        // The descriptor of the next pass is fetched while the current one runs.
+        int2 pd_next = p0 < p1 ? __ldg(reinterpret_cast<const int2 *>(args.passes + p0)) : make_int2(0, 0);
         for (int p = p0; p < p1; ++p) {
-            const int2 pd = __ldg(reinterpret_cast<const int2 *>(args.passes + p));
+            const int2 pd = pd_next;
+            if (p + 1 < p1) pd_next = __ldg(reinterpret_cast<const int2 *>(args.passes + p + 1));
             run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
                                         args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
         }
@@ -660,8 +666,11 @@ __global__ void __launch_bounds__(kWarpKernelThreads, MINB) spdy_forward_warp_ke
         for (int i = lane; i < ld.extent; i += 32) cur[i] = __int_as_float(0x7fc00000);
         __syncwarp();
 #endif
+        // The descriptor of the next pass is fetched while the current one runs.
+        int2 pd_next = p0 < p1 ? __ldg(reinterpret_cast<const int2 *>(args.passes + p0)) : make_int2(0, 0);
         for (int p = p0; p < p1; ++p) {
-            const int2 pd = __ldg(reinterpret_cast<const int2 *>(args.passes + p));
+            const int2 pd = pd_next;
+            if (p + 1 < p1) pd_next = __ldg(reinterpret_cast<const int2 *>(args.passes + p + 1));
             run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
                                         args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
         }
@@ -712,6 +721,8 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
     namespace cg = cooperative_groups;
     constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
     constexpr int NWARPS = NT / 32;
+    constexpr int CAP = NT >= 512 ? 16 : kRmax;  // == cluster_cells_per_lane(NT), the host's figure
+    static_assert(CAP <= kRmax, "pass bodies exist up to kRmax cells per lane");
     const FwdArgs &args = cargs.f;
     cg::cluster_group cluster = cg::this_cluster();
     const int C = cargs.C;
@@ -800,7 +811,7 @@ __global__ void __launch_bounds__(NT, 1) spdy_forward_cluster_kernel(const Clust
         switch (sd.cpl) {
 #define SPDY_CASE(RR)                                                                                             \
     case RR:                                                                                                      \
-        if constexpr (RR <= kRmax)                                                                                \
+        if constexpr (RR <= CAP)                                                                                  \
             for (int span = warp; span < sd.nspans; span += NWARPS) {                                             \
                 const int p = sd.mask_off + span;                                                                 \
                 const int2 pd = __ldg(reinterpret_cast<const int2 *>(args.passes + p));                           \
@@ -918,9 +929,12 @@ template <int MODE> constexpr int ctas_256() { return MODE == MODE_ARG_PAIR ? 2 
     SPDY_CTA_VARIANT(MODE, 512, 1, 8), SPDY_CTA_VARIANT(MODE, 1024, 1, 8)
 #define SPDY_FULL_VARIANTS(MODE)                                                                                \
     SPDY_CTA_VARIANTS(MODE),                                                                                    \
-    FwdVariant{KERNEL_CTA_GLOBAL, MODE, 1024, 12, spdy_forward_kernel<MODE, 1024, 1, 12, true>},                \
+    FwdVariant{KERNEL_CTA_GLOBAL, MODE, 1024, global_rows_cap_1024(MODE),                                       \
+               spdy_forward_kernel<MODE, 1024, 1, global_rows_cap_1024(MODE), true>},                           \
+    FwdVariant{KERNEL_CTA_GLOBAL, MODE, 512, kRmax, spdy_forward_kernel<MODE, 512, 1, kRmax, true>},            \
     FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, 8, spdy_forward_warp_kernel<MODE, 8, 8>},                 \
-    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, 16, spdy_forward_warp_kernel<MODE, 5, 16>},               \
+    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, warp_mid_cap(MODE),                                       \
+               spdy_forward_warp_kernel<MODE, 6, warp_mid_cap(MODE)>},                                          \
     FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, kRmax, spdy_forward_warp_kernel<MODE, 4, kRmax>}
 #define SPDY_CLUSTER_VARIANTS(MODE) \
     ClusterVariant{MODE, 256, spdy_forward_cluster_kernel<MODE, 256>}, ClusterVariant{MODE, 512, spdy_forward_cluster_kernel<MODE, 512>}

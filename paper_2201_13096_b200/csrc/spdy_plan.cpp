@@ -153,7 +153,7 @@ void build_slots(spdy_plan *p, int merge)
 // global memory the addresses are 64-bit, which costs a few more registers still.
 int cells_per_lane_cap(int kind, int threads, int mode)
 {
-    if (kind == KERNEL_CTA_GLOBAL) return 12;
+    if (kind == KERNEL_CTA_GLOBAL) return threads >= 1024 ? global_rows_cap_1024(mode) : kRmax;
     if (kind == KERNEL_WARP) return kRmax;
     return threads >= 1024 ? cells_per_lane_1024(mode) : kRmax;
 }
@@ -161,10 +161,13 @@ int cells_per_lane_cap(int kind, int threads, int mode)
 // The kernel builds differ in the largest pass they unroll; a plan picks the smallest that holds its passes.
 int rcap_for(int kind, int threads, int mode, int max_cpl)
 {
-    if (kind == KERNEL_CTA_GLOBAL) return 12;
-    if (kind == KERNEL_WARP) return max_cpl <= 8 ? 8 : (max_cpl <= 16 ? 16 : kRmax);
+    if (kind == KERNEL_CTA_GLOBAL) return cells_per_lane_cap(kind, threads, mode);
+    if (kind == KERNEL_WARP) return max_cpl <= 8 ? 8 : (max_cpl <= warp_mid_cap(mode) ? warp_mid_cap(mode) : kRmax);
     return max_cpl <= 8 ? 8 : cells_per_lane_cap(kind, threads, mode);
 }
+
+// CTA size of the rows-in-global-memory kernel when the caller leaves it open.
+constexpr int kGlobalRowsThreads = 1024;
 
 // Room left under the per-CTA shared-memory limit for the kernels' small static arrays (reductions).
 constexpr int64_t kStaticSmemReserve = 1024;
@@ -405,10 +408,11 @@ int layout_cluster(spdy_plan *p, int threads, int C)
             const int64_t ws = hi - lo;
             int64_t cpl = 1, nspans = 0;
             if (ws > 0) {
-                const int64_t per_round = 32LL * nwarps * kRmax;
+                const int64_t cap = cluster_cells_per_lane(threads);
+                const int64_t per_round = 32LL * nwarps * cap;
                 const int64_t rounds = (ws + per_round - 1) / per_round;
                 cpl = (ws + 32LL * nwarps * rounds - 1) / (32LL * nwarps * rounds);
-                cpl = std::min<int64_t>(kRmax, std::max<int64_t>(1, cpl));
+                cpl = std::min<int64_t>(cap, std::max<int64_t>(1, cpl));
                 nspans = (ws + 32 * cpl - 1) / (32 * cpl);
             }
             const int64_t span = 32 * cpl;
@@ -450,7 +454,7 @@ int layout_cluster(spdy_plan *p, int threads, int C)
     p->row_stride = 0;
     p->pad = 0;
     p->warps_per_cand = nwarps;
-    p->rcap = kRmax;
+    p->rcap = cluster_cells_per_lane(threads);
     p->smem_bytes = (2LL * p->out_stride + p->win_stride) * 4 + 2LL * ((p->K + 1) & ~1) * 8;
     return SPDY_OK;
 }
@@ -480,9 +484,8 @@ int choose_cluster_shape(spdy_plan *p, const spdy_options *opts)
 }
 
 // Wide-band fallback: one CTA of 1024 threads per candidate, row buffers in the workspace.
-int choose_global_row_shape(spdy_plan *p)
+int choose_global_row_shape(spdy_plan *p, int threads)
 {
-    const int threads = 1024;
     if (threads < p->K) return SPDY_ERR_UNSUPPORTED;
     p->mode = p->table_format == SPDY_TABLE_ARG_U8 ? MODE_ARG_PAIR : MODE_ROW2;  // the builds this shape has
     p->cluster = 1;
@@ -513,8 +516,8 @@ bool warp_kernel_fits(const spdy_plan *p)
                                 : (max_slots <= 64 && p->mode == MODE_ARG_PAIR);
 }
 
-// The warp kernel's builds unroll passes of up to 24, 16 or 8 cells per lane and need about 126, 96 and 64
-// registers per thread, which lets 4, 5 and 8 CTAs of 128 threads share an SM.  Longer passes are cheaper
+// The warp kernel's builds unroll passes of up to 24, warp_mid_cap() or 8 cells per lane in 128, 80 and 64
+// registers per thread, which lets 4, 6 and 8 CTAs of 128 threads share an SM.  Longer passes are cheaper
 // per cell, but only while registers do not cost resident warps that shared memory would allow: take the
 // longest pass whose register limit is no tighter than the shared-memory limit.
 int choose_warp_shape(spdy_plan *p)
@@ -525,7 +528,7 @@ int choose_warp_shape(spdy_plan *p)
     if (rc != SPDY_OK) return rc;
     if (asked_cap == 0) {
         const int by_smem = std::min(8, resident_ctas(p, threads, p->smem_bytes));
-        const int caps[3] = {kRmax, 16, 8}, by_regs[3] = {4, 5, 8};
+        const int caps[3] = {kRmax, warp_mid_cap(p->mode), 8}, by_regs[3] = {4, 6, 8};
         for (int i = 0; i < 3; ++i)
             if (by_regs[i] >= by_smem || i == 2) {
                 if (caps[i] < p->rcap) {
@@ -572,7 +575,8 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
         return SPDY_ERR_INVALID_ARG;
     if (opts && opts->rows_in_global) {
         if (opts->cluster > 1 || want_kernel == SPDY_KERNEL_WARP) return SPDY_ERR_INVALID_ARG;
-        return choose_global_row_shape(p);
+        if (opts->threads && opts->threads != 512 && opts->threads != 1024) return SPDY_ERR_INVALID_ARG;
+        return choose_global_row_shape(p, opts->threads ? opts->threads : kGlobalRowsThreads);
     }
     if (opts && opts->cluster > 1) {
         if (want_kernel == SPDY_KERNEL_WARP) return SPDY_ERR_INVALID_ARG;
@@ -609,9 +613,9 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
         // Rows in global memory, read through L1, measured faster than a cluster for such widths
         // (B = 10^5: 1.6x, B = 2*10^5: 1.9x) and have no width limit.  A cluster is still used when the
         // caller asks for one (cluster > 1, handled above) or pins a launch shape the fallback lacks.
-        if (opts && ((opts->threads && opts->threads != 1024) || opts->forward_mode))
+        if (opts && ((opts->threads && opts->threads != kGlobalRowsThreads) || opts->forward_mode))
             return choose_cluster_shape(p, opts);
-        return choose_global_row_shape(p);
+        return choose_global_row_shape(p, kGlobalRowsThreads);
     }
     // Narrow rows: a warp per candidate, unless the caller pinned a CTA shape.
     if (want_kernel == SPDY_KERNEL_AUTO && !(opts && opts->threads) && warp_kernel_fits(p) &&
@@ -846,12 +850,9 @@ const spdy_plan *pick_for_batch(const spdy_plan *p, int64_t N, size_t workspace_
             if (N * alt->cluster > p->limits.sm_count) continue;
             if (best->kind != KERNEL_CLUSTER || alt->cluster > best->cluster) best = alt;
         } else if (best->kind != KERNEL_CLUSTER) {
-            // A larger CTA per candidate while the batch leaves SMs under-filled: the largest CTA whose
-            // resident warps per SM do not exceed what the main shape would have at full load.
-            const int64_t ctas_per_sm_needed = (N + p->limits.sm_count - 1) / p->limits.sm_count;
-            if (ctas_per_sm_needed * alt->threads <= 1024 && ctas_per_sm_needed <= alt->ctas_per_sm &&
-                alt->threads > best->threads)
-                best = alt;
+            // A larger CTA per candidate when every candidate can have an SM to itself (measured: with two
+            // or more candidates per SM the main shape's longer passes per warp win again).
+            if (N <= p->limits.sm_count && alt->threads > best->threads) best = alt;
         }
     }
     return best;

@@ -19,8 +19,9 @@ constexpr int kLibraryVersion = 2000;
 // Most band cells one lane owns in one warp pass; the kernels unroll passes of 1..kRmax cells per lane.
 constexpr int kRmax = 24;
 
-// Widest band (cells) for which the plan prefers one warp per candidate when left to choose.
-constexpr int kWarpKernelMaxWidth = 1024;
+// Widest band (cells) for which the plan considers one warp per candidate when left to choose (it then
+// takes it if at least three CTAs of four candidates fit an SM).
+constexpr int kWarpKernelMaxWidth = 4096;
 
 // How the forward kernel forms a cell and what it stores for the walk back.
 enum ForwardMode {
@@ -34,6 +35,18 @@ enum ForwardMode {
 // Longest pass (cells per lane) a 1024-thread CTA unrolls: 64 registers per thread bound it, and the pairwise
 // argmin update keeps two register arrays per cell.
 constexpr int cells_per_lane_1024(int mode) { return mode == MODE_ARG_PAIR ? 8 : 16; }
+
+// Longest pass of a cluster's CTA: a 512-thread CTA has 128 registers per thread, which the masked stores of
+// a slice plus 24 cells per lane exceed.
+constexpr int cluster_cells_per_lane(int threads) { return threads >= 512 ? 16 : kRmax; }
+
+// Longest pass of the 1024-thread kernel whose rows live in global memory (64 registers per thread, 64-bit
+// row addresses).
+constexpr int global_rows_cap_1024(int mode) { return mode == MODE_ARG_PAIR ? 8 : 10; }
+
+// The warp-per-candidate kernel comes in three builds: passes of up to 8 cells per lane in 64 registers
+// (8 CTAs of 128 threads per SM), up to warp_mid_cap() in 80 registers (6 CTAs), up to kRmax in 128 (4 CTAs).
+constexpr int warp_mid_cap(int mode) { return mode == MODE_ARG_PAIR ? 12 : 18; }
 
 inline bool mode_is_row(int mode) { return mode == MODE_ROW || mode == MODE_ROW2; }
 inline bool mode_is_arg(int mode) { return mode == MODE_ARG || mode == MODE_ARG_PRED || mode == MODE_ARG_PAIR; }
