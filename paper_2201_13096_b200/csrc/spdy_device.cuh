@@ -199,25 +199,23 @@ __device__ __forceinline__ void update_arg(float (&best)[RR], int (&idx)[RR], co
     }
 }
 
-// Two slots k0 < k1 per step with the winning index read off the outcome: m = min(best, v0, v1); the cell
-// changes hands only if m < best (strict: a tie with the old value keeps the old, lower index), and then
-// to k0 if v0 attains m (a tie between the two goes to the lower index) and to k1 otherwise.  This is what
-// the scan "k0, then k1, strict <" leaves, at 2.5 instructions per update on top of load and add instead
-// of 3.  (A NaN sum never attains the minimum and never compares equal, as in the scan.)  A form that keeps
-// the index as a float and moves it under a predicate on the fp32 pipe (set, subtract, compare, predicated
-// add) has the same instruction count, loads the compare pipe less and measured 5 % slower.
+// Two slots k0 < k1 = k0 + 1 per step, the winner between the two left open: m = min(best, v0, v1); the cell
+// changes hands only if m < best (strict: a tie with the old value keeps the old, lower index), and then the
+// cell remembers the pair, not the slot: code = 2 * k0 + 1.  Which of the pair it was is settled once per
+// pass, after all slots (resolve_pair_codes).  Per update that is half a minimum, half a compare and half
+// a select on top of load and add - against a compare and two selects for the plain scan.  (A NaN sum never
+// attains the minimum, as in the scan.)
 template <int RR>
-__device__ __forceinline__ void update_arg_pair(float (&best)[RR], int (&idx)[RR], const Src sa, const float ea,
-                                                const int k0, const Src sb, const float eb, const int k1,
+__device__ __forceinline__ void update_arg_pair(float (&best)[RR], int (&code)[RR], const Src sa, const float ea,
+                                                const Src sb, const float eb, const int pair_code,
                                                 const AccessWindow &w)
 {
     const unsigned long long ea2 = splat2(ea), eb2 = splat2(eb);
-#define SPDY_PAIR_UPDATE(J, V0, V1)                     \
-    {                                                   \
-        const float m = min3(best[J], V0, V1);          \
-        const int kk = (V0 == m) ? k0 : k1;             \
-        idx[J] = (m < best[J]) ? kk : idx[J];           \
-        best[J] = m;                                    \
+#define SPDY_PAIR_UPDATE(J, V0, V1)                         \
+    {                                                       \
+        const float m = min3(best[J], V0, V1);              \
+        code[J] = (m < best[J]) ? pair_code : code[J];      \
+        best[J] = m;                                        \
     }
 #pragma unroll
     for (int j = 0; j + 1 < RR; j += 2) {
@@ -234,6 +232,27 @@ __device__ __forceinline__ void update_arg_pair(float (&best)[RR], int (&idx)[RR
         SPDY_PAIR_UPDATE(RR - 1, a0, b0);
     }
 #undef SPDY_PAIR_UPDATE
+}
+
+// Codes of update_arg_pair -> slot indices, once per pass.  A cell whose code names a pair (odd) won with
+// m = min(v0, v1) of that pair and nothing after it was smaller, so best still holds that m: the winner is
+// k0 if v0 - the same fp32 add of the same operands, hence the same bits - equals best, else k1 (a tie
+// between the two goes to the lower index, as in the scan).  An even code 2 * k names slot k itself (slots
+// taken singly); the initial code names no slot (0xFF).
+template <int RR>
+__device__ __forceinline__ void resolve_pair_codes(const float (&best)[RR], int (&code)[RR], const float *prev,
+                                                   const int2 *taps, const int first, const int k_any,
+                                                   const AccessWindow &w)
+{
+#pragma unroll
+    for (int j = 0; j < RR; ++j) {
+        const int c = code[j];
+        const bool pair = c & 1;
+        const int k0 = c >> 1;
+        const int2 tp = taps[pair ? k0 : k_any];  // k_any: some slot of this pass, so that every lane reads in range
+        const float v0 = __fadd_rn(make_src(prev, first, tp.x).at(j, w), __int_as_float(tp.y));
+        code[j] = (pair && !(v0 == best[j])) ? k0 + 1 : k0;
+    }
 }
 
 // Same update as update_arg with the two selects written as predicated fp32 arithmetic that acts as an exact
@@ -351,28 +370,13 @@ __device__ __forceinline__ void process_span(const float *prev, float *cur, cons
 #pragma unroll
         for (int j = 0; j < RR; ++j)
             if (store_allowed(j)) D[j * 32] = best[j];
-    } else if constexpr (MODE == MODE_ARG || MODE == MODE_ARG_PAIR) {
+    } else if constexpr (MODE == MODE_ARG) {
         int idx[RR];
 #pragma unroll
         for (int j = 0; j < RR; ++j) idx[j] = 0xFF;
         if (dense) {
-            int k = k_lo;
-            if (MODE == MODE_ARG_PAIR) {
-                // An odd first slot goes alone so that every pair below is one aligned 16-byte read.
-                if ((k & 1) && k < k_hi) {
-                    const int2 tp = taps[k];
-                    update_arg<RR>(best, idx, make_src(prev, first, tp.x), __int_as_float(tp.y), k, w);
-                    ++k;
-                }
 #pragma unroll 1
-                for (; k + 1 < k_hi; k += 2) {
-                    const int4 t = *reinterpret_cast<const int4 *>(taps + k);
-                    update_arg_pair<RR>(best, idx, make_src(prev, first, t.x), __int_as_float(t.y), k,
-                                        make_src(prev, first, t.z), __int_as_float(t.w), k + 1, w);
-                }
-            }
-#pragma unroll 1
-            for (; k < k_hi; ++k) {
+            for (int k = k_lo; k < k_hi; ++k) {
                 const int2 tp = taps[k];
                 update_arg<RR>(best, idx, make_src(prev, first, tp.x), __int_as_float(tp.y), k, w);
             }
@@ -396,6 +400,51 @@ __device__ __forceinline__ void process_span(const float *prev, float *cur, cons
 #pragma unroll
         for (int j = 0; j < RR; ++j)
             if (store_allowed(j)) P[j * 32] = static_cast<unsigned char>(idx[j]);
+    } else if constexpr (MODE == MODE_ARG_PAIR) {
+        // code: 2 * k for "slot k", 2 * k0 + 1 for "slot k0 or k0 + 1" (settled below), 2 * 0xFF for none.
+        int code[RR];
+#pragma unroll
+        for (int j = 0; j < RR; ++j) code[j] = 2 * 0xFF;
+        if (dense) {
+            int k = k_lo;
+            // An odd first slot goes alone so that every pair below is one aligned 16-byte read.
+            if ((k & 1) && k < k_hi) {
+                const int2 tp = taps[k];
+                update_arg<RR>(best, code, make_src(prev, first, tp.x), __int_as_float(tp.y), 2 * k, w);
+                ++k;
+            }
+#pragma unroll 1
+            for (; k + 1 < k_hi; k += 2) {
+                const int4 t = *reinterpret_cast<const int4 *>(taps + k);
+                update_arg_pair<RR>(best, code, make_src(prev, first, t.x), __int_as_float(t.y),
+                                    make_src(prev, first, t.z), __int_as_float(t.w), 2 * k + 1, w);
+            }
+            if (k < k_hi) {
+                const int2 tp = taps[k];
+                update_arg<RR>(best, code, make_src(prev, first, tp.x), __int_as_float(tp.y), 2 * k, w);
+            }
+            if (k_lo < k_hi) resolve_pair_codes<RR>(best, code, prev, taps, first, k_lo, w);
+        } else {
+#pragma unroll 1
+            for (int wd = 0; wd < MW; ++wd) {
+                unsigned long long m = __ldg(mask + wd);
+#pragma unroll 1
+                while (m) {
+                    const int k = 64 * wd + __ffsll(static_cast<long long>(m)) - 1;
+                    m &= m - 1;
+                    const int2 tp = taps[k];
+                    update_arg<RR>(best, code, make_src(prev, first, tp.x), __int_as_float(tp.y), 2 * k, w);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < RR; ++j)
+            if (store_allowed(j)) cur[s + j * 32 + lane] = best[j];
+        unsigned char *P = static_cast<unsigned char *>(table_row) + s + lane;
+        // (dense passes hold slot indices after resolve_pair_codes, the others still 2 * k)
+#pragma unroll
+        for (int j = 0; j < RR; ++j)
+            if (store_allowed(j)) P[j * 32] = static_cast<unsigned char>(dense && k_lo < k_hi ? code[j] : code[j] >> 1);
     } else {  // MODE_ARG_PRED
         float idxf[RR];
 #pragma unroll
