@@ -530,9 +530,11 @@ def run_sweep(args):
                      and np.array_equal(t[sample], ref[2]))
         cellb = 4 if info["table_format"] == 2 else 1
         hbm_bytes = wl.N * (info["band_cells"] * cellb + wl.L * wl.K * 4)
+        shape = plan.shape_for_batch(wl.N, ws.numel())  # small batches run on a launch shape of their own
         row = {"workload": wl.name, "N": wl.N, "L": wl.L, "K": wl.K, "B": wl.B,
                "table_format": {1: "arg_u8", 2: "row_f32"}[info["table_format"]],
-               "threads": info["threads"], "cluster": info["cluster"], "rows_in_global": info["rows_in_global"],
+               "threads": shape["threads"], "cluster": shape["cluster"], "rows_in_global": info["rows_in_global"],
+               "warp_per_candidate": int(shape["kernel_kind"] == 3),
                "gpu_ms": ms, "forward_ms": f_ms, "walkback_ms": float(np.mean(back)),
                "candidates_per_s": wl.N / (ms * 1e-3),
                "nominal_cell_updates_per_s": wl.N * info["nominal_updates"] / (ms * 1e-3),
@@ -552,7 +554,8 @@ def run_sweep(args):
     print(head, file=sys.stderr)
     print("|" + "---|" * 12, file=sys.stderr)
     for r in rows:
-        shape = f'{r["threads"]} thr' + (f' x{r["cluster"]}' if r["cluster"] > 1 else "") + (", rows in global" if r["rows_in_global"] else "")
+        shape = (f'{r["threads"]} thr' + (f' x{r["cluster"]}' if r["cluster"] > 1 else "")
+                 + (", rows in global" if r["rows_in_global"] else "") + (", warp per candidate" if r["warp_per_candidate"] else ""))
         print(f'| {r["workload"]} | {r["table_format"]} | {shape} | {r["gpu_ms"]:.3f} | {r["candidates_per_s"]:.4g} | '
               f'{r["nominal_cell_updates_per_s"]:.3g} | {r["executed_cell_updates_per_s"]:.3g} | '
               f'{r["roofline_frac_of_measured_lds"]:.3f} | {r["table_and_errors_gb_per_s"]:.0f} | '

@@ -198,6 +198,11 @@ typedef struct spdy_plan_tables {
     const int32_t *slices;
 } spdy_plan_tables;
 int spdy_plan_get_tables(const spdy_plan *plan, int32_t which, spdy_plan_tables *out);
+
+/* Which table set spdy_solve_batch would run a batch of N candidates on, given `workspace_bytes` of
+ * workspace: 0 = the main launch shape, i >= 1 = the i-th launch shape for small batches (the index
+ * spdy_plan_get_tables takes).  Returns -1 for a null plan. */
+int32_t spdy_plan_shape_for_batch(const spdy_plan *plan, int64_t N, size_t workspace_bytes);
 int spdy_plan_verify(const spdy_plan *plan);
 
 /* The walk-back table is Algorithm 1's L x (T+1) matrix (the O(L*T) memory of Section 3.2), kept per

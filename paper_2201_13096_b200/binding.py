@@ -29,11 +29,12 @@ EXPORTS = (
     "spdy_solve_batch_coeffs", "spdy_solve_batch_coeffs_host", "spdy_quadratic_errors",
     "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile", "spdy_probe_peaks",
     "spdy_plan_get_tables", "spdy_plan_verify", "spdy_plan_status_word", "spdy_debug_checks_enabled",
+    "spdy_plan_shape_for_batch",
 )
 # What the host-only library holds (everything that needs no CUDA).
 HOST_EXPORTS = (
     "spdy_plan_create", "spdy_plan_destroy", "spdy_plan_get_info", "spdy_plan_get_bands", "spdy_workspace_bytes",
-    "spdy_plan_get_tables", "spdy_plan_verify", "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile",
+    "spdy_plan_get_tables", "spdy_plan_verify", "spdy_plan_shape_for_batch", "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile",
     "spdy_strerror", "spdy_version",
 )
 
@@ -101,6 +102,8 @@ def _configure(lib, host_only: bool = False):
     lib.spdy_plan_get_tables.argtypes = [vp, i32, ctypes.POINTER(SpdyPlanTables)]
     lib.spdy_plan_verify.restype = ctypes.c_int
     lib.spdy_plan_verify.argtypes = [vp]
+    lib.spdy_plan_shape_for_batch.restype = ctypes.c_int32
+    lib.spdy_plan_shape_for_batch.argtypes = [vp, i64, ctypes.c_size_t]
     lib.spdy_workspace_bytes.restype = ctypes.c_size_t
     lib.spdy_workspace_bytes.argtypes = [vp, i64]
     lib.spdy_time_target.restype = ctypes.c_double
@@ -263,6 +266,15 @@ class Plan:
         out["pass_ptr"] = arr(t.pass_ptr, ctypes.c_int32, (out["L"] * W + 1,)) if t.pass_ptr else None
         out["slices"] = arr(t.slices, ctypes.c_int32, (out["L"], out["cluster"], 8)) if t.slices else None
         return out
+
+    def shape_for_batch(self, N: int, workspace_bytes: Optional[int] = None) -> dict:
+        """The launch shape ``spdy_solve_batch`` would use for N candidates (``spdy_plan_shape_for_batch``):
+        kernel kind, threads per CTA, CTAs per candidate, and the table-set index."""
+        ws = self.workspace_bytes(N) if workspace_bytes is None else int(workspace_bytes)
+        which = int(_load().spdy_plan_shape_for_batch(self._h, int(N), ws))
+        t = SpdyPlanTables()
+        _check(_load().spdy_plan_get_tables(self._h, which, ctypes.byref(t)), "spdy_plan_get_tables")
+        return {"which": which, "kernel_kind": int(t.kernel_kind), "threads": int(t.threads), "cluster": int(t.cluster)}
 
     def status_word(self, stream=None) -> int:
         """``spdy_plan_status_word``: read and clear the self-check word (0 = nothing flagged)."""

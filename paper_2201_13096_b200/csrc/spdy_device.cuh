@@ -598,13 +598,22 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         for (int i = tid; i < ld.extent; i += NT) cur[i] = __int_as_float(0x7fc00000);  // mark the new row unwritten
         __syncthreads();
 #endif
-        // The descriptor of the next pass is fetched while the current one runs.
-        int2 pd_next = p0 < p1 ? __ldg(reinterpret_cast<const int2 *>(args.passes + p0)) : make_int2(0, 0);
-        for (int p = p0; p < p1; ++p) {
-            const int2 pd = pd_next;
-            if (p + 1 < p1) pd_next = __ldg(reinterpret_cast<const int2 *>(args.passes + p + 1));
-            run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
-                                        args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
+        if constexpr (GROWS) {
+            // (64 registers per thread: no room to hold the next pass's descriptor across a pass)
+            for (int p = p0; p < p1; ++p) {
+                const int2 pd = __ldg(reinterpret_cast<const int2 *>(args.passes + p));
+                run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+                                            args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
+            }
+        } else {
+            // The descriptor of the next pass is fetched while the current one runs.
+            int2 pd_next = p0 < p1 ? __ldg(reinterpret_cast<const int2 *>(args.passes + p0)) : make_int2(0, 0);
+            for (int p = p0; p < p1; ++p) {
+                const int2 pd = pd_next;
+                if (p + 1 < p1) pd_next = __ldg(reinterpret_cast<const int2 *>(args.passes + p + 1));
+                run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+                                            args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
+            }
         }
         // Cells [width, extent) of the new row were written as +inf by the passes (they saw only +inf
         // sources); PAD more cells of +inf behind them cover every read of the next layer.

@@ -1072,6 +1072,15 @@ int spdy_plan_get_tables(const spdy_plan *plan, int32_t which, spdy_plan_tables 
     return SPDY_OK;
 }
 
+int32_t spdy_plan_shape_for_batch(const spdy_plan *plan, int64_t N, size_t workspace_bytes)
+{
+    if (!plan) return -1;
+    const spdy_plan *shape = pick_for_batch(plan, N, workspace_bytes);
+    for (size_t i = 0; i < plan->alternates.size(); ++i)
+        if (plan->alternates[i] == shape) return static_cast<int32_t>(i + 1);
+    return 0;
+}
+
 int spdy_plan_verify(const spdy_plan *plan)
 {
     if (!plan) return SPDY_ERR_INVALID_ARG;

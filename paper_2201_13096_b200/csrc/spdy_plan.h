@@ -14,7 +14,7 @@
 
 namespace spdy {
 
-constexpr int kLibraryVersion = 2000;
+constexpr int kLibraryVersion = 2001;
 
 // Most band cells one lane owns in one warp pass; the kernels unroll passes of 1..kRmax cells per lane.
 constexpr int kRmax = 24;
@@ -42,7 +42,7 @@ constexpr int cluster_cells_per_lane(int threads) { return threads >= 512 ? 16 :
 
 // Longest pass of the 1024-thread kernel whose rows live in global memory (64 registers per thread, 64-bit
 // row addresses).
-constexpr int global_rows_cap_1024(int mode) { return mode == MODE_ARG_PAIR ? 8 : 10; }
+constexpr int global_rows_cap_1024(int mode) { return mode == MODE_ARG_PAIR ? 8 : 12; }
 
 // The warp-per-candidate kernel comes in three builds: passes of up to 8 cells per lane in 64 registers
 // (8 CTAs of 128 threads per SM), up to warp_mid_cap() in 80 registers (6 CTAs), up to kRmax in 128 (4 CTAs).
