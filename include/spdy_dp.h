@@ -94,11 +94,13 @@ typedef struct spdy_options {
                               do not fit one CTA's shared memory (B of about 10^5 buckets and more); any width
                               runs.  One CTA of 1024 threads per candidate; not combinable with cluster > 1 */
     int32_t kernel;        /* spdy_kernel */
-    int32_t schedule;      /* how a row is cut into warp passes.  Bits 0-7: 0 = passes of one length per layer,
-                              dealt round-robin (default); 1 = passes sized by the slots that overlap them
-                              and dealt to the warps by cost (fewer cell updates issued, measured slower; for
-                              measurement).  Bits 8-15: upper limit of cells per lane per pass, 1..24
-                              (0 = the kernel's own limit; for measurement) */
+    int32_t schedule;      /* how a row is cut into warp passes.  Bits 0-7: 0 = the plan's choice (2 with the
+                              fp32 table, 1 with the uint8 table); 1 = passes of one length per layer, dealt
+                              round-robin; 2 = as many passes, cut where their costs are level (fewer updates
+                              wasted on slots that overlap a pass only partly); 3 = passes sized by dynamic
+                              programming and dealt to the warps by load (least waste, most passes, measured
+                              slowest; for measurement).  Bits 8-15: upper limit of cells per lane per pass,
+                              1..24 (0 = the kernel's own limit; for measurement) */
     int32_t auto_shape;    /* 0: when threads, cluster, rows_in_global and kernel are all 0 the plan also lays
                               out launch shapes for batches too small to fill the device (larger CTAs, clusters
                               of 2/4/8) and spdy_solve_batch picks by N; 1: never, one shape for every N */

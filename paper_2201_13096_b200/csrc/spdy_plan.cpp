@@ -179,15 +179,21 @@ struct PassPlan {
     double cost;
 };
 
-// Passes of one layer.  `ba`/`bb`: first and last 32-cell block each slot touches.
-// schedule 0 (default): passes of one length, chosen so that the rounds of W passes are equally full, dealt
-// round-robin: every warp runs the same unrolled body and the warps arrive level at the layer's barrier.
-// schedule 1: pass boundaries by dynamic programming over the blocks, minimising issued work - a pass is
-// all-or-nothing per slot, so a slot that overlaps it only partly costs the whole pass; short passes where
-// slots begin and end (the ramps at both ends of a band), long ones in between - then dealt to the warps
-// longest first onto the least loaded warp; the pass length cap shrinks until the warps are level within a few
-// per cent.  It issues 3 % fewer cell updates at the BERT-base shape and measured 1.5 % slower there (11 %
-// slower with rows in global memory): the passes of mixed lengths cost more than the updates they save.
+// Passes of one layer.  `ba`/`bb`: first and last 32-cell block each slot touches.  A pass is all-or-nothing
+// per slot: a slot that overlaps it only partly costs the whole pass.
+// SCHED_UNIFORM: passes of one length, chosen so that the rounds of W passes are equally full, dealt
+// round-robin: every warp runs the same unrolled body.
+// SCHED_LEVELLED: as many passes as that, but cut where their costs (in shared-memory wavefronts) are
+// level: a pass over the ramp at either end of a band, where few slots overlap, is longer or shorter than
+// one in the middle so that all cost the same, which both trims the partly overlapping work (4.5 % -> 2.6 %
+// of the issued updates at the BERT-base shape) and keeps the warps level at the layer's barrier.
+// SCHED_SIZED: pass boundaries by dynamic programming over the blocks, minimising the summed cost (short
+// passes where slots begin and end, long ones in between), then dealt to the warps longest first onto the
+// least loaded warp, the pass length cap shrinking until the warps are level within a few per cent.  It
+// wastes least (1.6 %) and measures slowest: it makes half as many passes again, and every pass pays for its
+// own slot reads and set-up.  One warp per candidate has nobody to level with and takes it as its LEVELLED.
+constexpr int SCHED_UNIFORM = 1, SCHED_LEVELLED = 2, SCHED_SIZED = 3;
+
 void plan_layer_passes(const std::vector<int> &ba, const std::vector<int> &bb, int nb, int W, int R, int schedule,
                        std::vector<std::vector<PassPlan>> &per_warp, double *total_cost, double *makespan,
                        int *blocks_covered)
@@ -208,11 +214,12 @@ void plan_layer_passes(const std::vector<int> &ba, const std::vector<int> &bb, i
         ended[j] += ended[j - 1];
     }
     auto overlapping = [&](int i, int j) { return started[std::min(j, nb + 1)] - ended[std::min(i, nb + 1)]; };
-    // Issue cost of a pass in units of one warp-wide cell update: the updates themselves, one 16-byte slot
-    // read per two slots, the stores of the new row (shared memory and table), and the loop set-up.
+    // Cost of a pass in wavefronts of the shared-memory data path, the unit the kernel is bound by: one per
+    // slot and 32 cells, the 16-byte slot-pair reads (two wavefronts per pair), the stores of the new row
+    // (shared memory and table), and the pass's own descriptor and set-up.
     auto pass_cost = [&](int i, int j) {
         const int n = overlapping(i, j);
-        return static_cast<double>(n) * ((j - i) + 0.5) + 2.0 * (j - i) + 8.0;
+        return static_cast<double>(n) * ((j - i) + 1.0) + 2.3 * (j - i) + 6.0;
     };
     auto finish = [&](std::vector<PassPlan> &passes) {
         for (PassPlan &pp : passes) {
@@ -252,7 +259,7 @@ void plan_layer_passes(const std::vector<int> &ba, const std::vector<int> &bb, i
     };
 
     std::vector<PassPlan> passes;
-    if (schedule == 0) {
+    if (schedule == SCHED_UNIFORM) {
         const int64_t per_round = static_cast<int64_t>(W) * R;
         const int64_t rounds = std::max<int64_t>(1, (nb + per_round - 1) / per_round);
         int64_t cpl = (nb + W * rounds - 1) / (W * rounds);
@@ -261,6 +268,60 @@ void plan_layer_passes(const std::vector<int> &ba, const std::vector<int> &bb, i
         *blocks_covered = passes.back().j;  // the last pass may run past the band; those cells hold +inf
         finish(passes);
         deal(passes, true);
+        return;
+    }
+    if (schedule == SCHED_LEVELLED && W > 1) {
+        // Levelled partition: for one, two or three more rounds than the row needs, cut the blocks into
+        // W * rounds contiguous passes whose largest cost is as small as possible (binary search on that
+        // bottleneck; a pass is extended while it stays under it), deal them round-robin, and keep the
+        // partition with the smallest load on the busiest warp - the uniform schedule included.
+        const int r0 = std::max(1, (nb + W * R - 1) / (W * R));
+        std::vector<PassPlan> best_passes;
+        double best_span = 1e300;
+        auto cut = [&](double bound, std::vector<PassPlan> *out) {
+            int count = 0;
+            for (int i = 0; i < nb;) {
+                int j = i + 1;
+                while (j < nb && j - i < R && pass_cost(i, j + 1) <= bound) ++j;
+                if (out) out->push_back(PassPlan{i, j, 0, 0, 0, 0.0});
+                ++count;
+                i = j;
+            }
+            return count;
+        };
+        for (int rounds = r0; rounds <= r0 + 2; ++rounds) {
+            const int P = std::min(nb, W * rounds);
+            double lo = 0.0, hi = pass_cost(0, std::min(nb, R)) * 2.0 + 1.0;
+            for (int i = 0; i < nb; ++i) lo = std::max(lo, pass_cost(i, i + 1));
+            if (cut(hi, nullptr) > P) continue;
+            for (int it = 0; it < 40; ++it) {
+                const double mid = 0.5 * (lo + hi);
+                if (cut(mid, nullptr) <= P) hi = mid;
+                else lo = mid;
+            }
+            std::vector<PassPlan> trial;
+            cut(hi, &trial);
+            finish(trial);
+            deal(trial, true);
+            if (*makespan < best_span) {
+                best_span = *makespan;
+                best_passes = trial;
+            }
+        }
+        {
+            const int64_t rounds = r0;
+            int64_t cpl = (nb + W * rounds - 1) / (W * rounds);
+            cpl = std::min<int64_t>(R, std::max<int64_t>(1, cpl));
+            std::vector<PassPlan> trial;
+            for (int i = 0; i < nb; i += static_cast<int>(cpl)) trial.push_back(PassPlan{i, static_cast<int>(std::min<int64_t>(nb, i + cpl)), 0, 0, 0, 0.0});
+            finish(trial);
+            deal(trial, true);
+            if (*makespan <= best_span) {
+                best_span = *makespan;
+                best_passes = trial;
+            }
+        }
+        deal(best_passes, true);
         return;
     }
     std::vector<double> best(nb + 1);
@@ -561,8 +622,11 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
     }
     p->schedule = opts ? (opts->schedule & 0xFF) : 0;
     p->pass_cap = opts ? ((opts->schedule >> 8) & 0xFF) : 0;
-    if (p->schedule < 0 || p->schedule > 1 || (opts && (opts->schedule >> 16) != 0) || p->pass_cap > kRmax)
+    if (p->schedule < 0 || p->schedule > SCHED_SIZED || (opts && (opts->schedule >> 16) != 0) || p->pass_cap > kRmax)
         return SPDY_ERR_INVALID_ARG;
+    // Left open: levelled passes where the shared-memory data path binds (row-value table); passes of one
+    // length where instruction issue binds (byte table: one unrolled body per layer measured 3 % faster).
+    if (p->schedule == 0) p->schedule = mode_is_row(p->mode) ? SCHED_LEVELLED : SCHED_UNIFORM;
     build_slots(p, mode_is_row(p->mode) ? 1 : (p->merge_first ? 2 : 0));
     p->cluster = 1;
     p->kind = KERNEL_CTA;

@@ -141,7 +141,7 @@ struct spdy_plan {
     int cluster = 1;
     int table_format = SPDY_TABLE_ROW_F32;
     int ctas_per_sm = 0;
-    int schedule = 0;        // 0 = passes of one length dealt round-robin, 1 = cost-sized passes dealt by load
+    int schedule = 0;        // resolved pass schedule: 1 uniform, 2 levelled, 3 cost-sized (see spdy_plan.cpp)
     int pass_cap = 0;        // upper limit of cells per lane per pass asked for by the options (0 = the kernel's)
     spdy::DeviceLimits limits;
     int64_t smem_bytes = 0;

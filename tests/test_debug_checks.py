@@ -41,7 +41,7 @@ def same(got, ref):
 
 SHAPES = [dict(), dict(kernel=binding.SPDY_KERNEL_WARP), dict(kernel=binding.SPDY_KERNEL_CTA), dict(threads=256),
           dict(threads=1024), dict(rows_in_global=1), dict(cluster=2), dict(cluster=8), dict(schedule=1),
-          dict(schedule=4 << 8)]
+          dict(schedule=3), dict(schedule=4 << 8)]
 
 
 @pytest.mark.parametrize("fmt", FORMATS)

@@ -536,7 +536,7 @@ def test_random_shapes_formats_and_launch_options():
         ref = oracle.solve_batch(wl.errors, wl.times, wl.B)
         options = [dict(), dict(cluster=int(rng.choice([2, 4, 8]))), dict(rows_in_global=1),
                    dict(threads=int(rng.choice([256, 512, 1024]))), dict(kernel=binding.SPDY_KERNEL_WARP),
-                   dict(kernel=binding.SPDY_KERNEL_CTA, schedule=1), dict(schedule=int(rng.integers(1, 9)) << 8)]
+                   dict(kernel=binding.SPDY_KERNEL_CTA, schedule=int(rng.integers(1, 4))), dict(schedule=int(rng.integers(1, 9)) << 8)]
         for fmt in FORMATS:
             kw = options[int(rng.integers(len(options)))]
             try:
@@ -631,10 +631,10 @@ def test_one_warp_per_candidate_gives_the_same_answer(fmt):
 
 @pytest.mark.parametrize("fmt", FORMATS)
 def test_pass_schedules_give_the_same_answer(fmt):
-    """Passes of one size dealt round-robin (default), passes sized by cost, and capped pass lengths."""
+    """The plan's choice, passes of one length, levelled passes, cost-sized passes, capped pass lengths."""
     wl = W.make_workload(2, N=6)
     ref = oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)
-    for schedule in (0, 1, 5 << 8, 1 | (3 << 8), 16 << 8):
+    for schedule in (0, 1, 2, 3, 5 << 8, 3 | (3 << 8), 2 | (16 << 8)):
         for threads in (128, 512):
             assert_same(gpu_solve(wl, fmt, schedule=schedule, threads=threads), ref)
 

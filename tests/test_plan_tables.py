@@ -152,9 +152,9 @@ def replay(t, times, errors_one, B, merged):
     return last[tt], int(layers[L - 1, 2]) + tt
 
 
-SHAPES = [dict(), dict(table_format=U8), dict(schedule=1), dict(threads=256), dict(threads=512), dict(threads=1024),
+SHAPES = [dict(), dict(table_format=U8), dict(schedule=1), dict(schedule=2), dict(schedule=3), dict(table_format=U8, schedule=2), dict(threads=256), dict(threads=512), dict(threads=1024),
           dict(rows_in_global=1), dict(kernel=binding.SPDY_KERNEL_WARP), dict(kernel=binding.SPDY_KERNEL_CTA),
-          dict(table_format=U8, kernel=binding.SPDY_KERNEL_WARP), dict(schedule=1 | (6 << 8)), dict(schedule=5 << 8),
+          dict(table_format=U8, kernel=binding.SPDY_KERNEL_WARP), dict(schedule=3 | (6 << 8)), dict(schedule=5 << 8),
           dict(cluster=2), dict(cluster=4), dict(cluster=8), dict(table_format=U8, cluster=4)]
 
 
@@ -207,7 +207,7 @@ def test_margins_and_replay_on_fuzzed_shapes():
             times[rng.integers(L), :] = 0
         errors = rng.lognormal(0.0, 1.0, size=(1, L, K)).astype(np.float32)
         ref = oracle.solve_batch(errors, times, B)
-        for kw in (dict(), dict(table_format=U8), dict(kernel=binding.SPDY_KERNEL_WARP), dict(schedule=1),
+        for kw in (dict(), dict(table_format=U8), dict(kernel=binding.SPDY_KERNEL_WARP), dict(schedule=1), dict(schedule=3),
                    dict(cluster=int(rng.choice([2, 4, 8]))), dict(rows_in_global=1)):
             plan, sets = plans_of(times, B, **kw)
             if plan is None:
@@ -224,7 +224,7 @@ def test_margins_and_replay_on_fuzzed_shapes():
 
 @pytest.mark.parametrize("cfg,B,kw", [(2, None, dict()), (2, None, dict(table_format=U8)), (1, None, dict()),
                                       (4, 1000, dict()), (4, 1000, dict(kernel=binding.SPDY_KERNEL_CTA)),
-                                      (4, 2500, dict(threads=256)), (2, None, dict(schedule=1))])
+                                      (4, 2500, dict(threads=256)), (2, None, dict(schedule=1)), (2, None, dict(schedule=3))])
 def test_replay_of_the_named_shapes_matches_the_oracle(cfg, B, kw):
     wl = W.make_workload(cfg, N=2, B=B)
     ref = oracle.solve_batch(wl.errors, wl.times, wl.B)
@@ -237,15 +237,21 @@ def test_replay_of_the_named_shapes_matches_the_oracle(cfg, B, kw):
             assert np.float32(cost).tobytes() == ref[1][n].tobytes() and tu == ref[2][n], (label, n)
 
 
-def test_cost_sized_passes_cut_the_issued_work():
-    """The cost-sized passes (schedule 1) issue fewer cell updates than passes of one size (a pass is
-    all-or-nothing per slot); the work that has to be done is the same."""
+def test_pass_schedules_trade_wasted_updates_against_passes():
+    """A pass is all-or-nothing per slot.  Passes of one length waste most updates on partly overlapping
+    slots, levelled passes (the default with the fp32 table) fewer with as many passes, cost-sized passes
+    fewest with half as many passes again; the work that has to be done is the same."""
     wl = W.make_workload(2, N=1)
-    sized = binding.Plan(wl.times, wl.B, device=-1, auto_shape=1, schedule=1).info
-    uniform = binding.Plan(wl.times, wl.B, device=-1, auto_shape=1).info
-    assert sized["distinct_updates"] == uniform["distinct_updates"]
-    assert sized["distinct_updates"] <= sized["issued_updates"] < uniform["issued_updates"]
-    assert sized["issued_updates"] < 1.03 * sized["distinct_updates"] < uniform["issued_updates"] < 1.06 * sized["distinct_updates"]
+    plans = {s: binding.Plan(wl.times, wl.B, device=-1, auto_shape=1, schedule=s) for s in (0, 1, 2, 3)}
+    info = {s: p.info for s, p in plans.items()}
+    passes = {s: p.tables(0)["n_passes"] for s, p in plans.items()}
+    assert len({i["distinct_updates"] for i in info.values()}) == 1
+    d = info[1]["distinct_updates"]
+    assert d <= info[3]["issued_updates"] < info[2]["issued_updates"] < info[1]["issued_updates"] < 1.06 * d
+    assert info[0]["issued_updates"] == info[2]["issued_updates"] < 1.03 * d
+    assert passes[2] <= 1.05 * passes[1] and passes[3] > 1.2 * passes[1]
+    u8 = binding.Plan(wl.times, wl.B, device=-1, auto_shape=1, table_format=U8).info
+    assert u8["issued_updates"] == info[1]["issued_updates"]  # the byte table keeps passes of one length
 
 
 def test_small_batches_get_their_own_launch_shapes():
