@@ -302,7 +302,10 @@ __device__ __forceinline__ void update_arg_pred(float (&best)[RR], float (&idxf)
 //
 // With MASKED only cells below `limit` are stored (a CTA of a cluster owns a slice of the band and
 // must not write its neighbour's cells); without it the caller guarantees room for the whole pass.
-template <int RR, int MODE, bool MASKED>
+//
+// With STORE_TABLE false (row-value table only) the pass leaves the table alone: the caller copies the whole
+// row from shared memory to the table with one bulk copy per layer.
+template <int RR, int MODE, bool MASKED, bool STORE_TABLE = true>
 __device__ __forceinline__ void process_span(const float *prev, float *cur, const int2 *__restrict__ taps,
                                              const unsigned krange, const unsigned long long *__restrict__ mask,
                                              const int MW, const int s, const int lane, void *table_row,
@@ -366,10 +369,12 @@ __device__ __forceinline__ void process_span(const float *prev, float *cur, cons
 #pragma unroll
         for (int j = 0; j < RR; ++j)
             if (store_allowed(j)) cur[s + j * 32 + lane] = best[j];
-        float *D = static_cast<float *>(table_row) + s + lane;
+        if constexpr (STORE_TABLE) {
+            float *D = static_cast<float *>(table_row) + s + lane;
 #pragma unroll
-        for (int j = 0; j < RR; ++j)
-            if (store_allowed(j)) D[j * 32] = best[j];
+            for (int j = 0; j < RR; ++j)
+                if (store_allowed(j)) D[j * 32] = best[j];
+        }
     } else if constexpr (MODE == MODE_ARG) {
         int idx[RR];
 #pragma unroll
@@ -479,7 +484,7 @@ __device__ __forceinline__ void process_span(const float *prev, float *cur, cons
 }
 
 // Runs the pass `pd` with the unrolled body for its cells-per-lane count (1..RCAP).
-template <int MODE, int RCAP, bool MASKED>
+template <int MODE, int RCAP, bool MASKED, bool STORE_TABLE = true>
 __device__ __forceinline__ void run_pass(const int cpl, const float *prev, float *cur, const int2 *taps,
                                          const unsigned krange, const unsigned long long *mask, const int MW,
                                          const int s, const int lane, void *table_row, const int limit,
@@ -489,7 +494,8 @@ __device__ __forceinline__ void run_pass(const int cpl, const float *prev, float
 #define SPDY_CASE(RR)                                                                                          \
     case RR:                                                                                                   \
         if constexpr (RR <= kRmax && RR <= RCAP)                                                               \
-            process_span<RR, MODE, MASKED>(prev, cur, taps, krange, mask, MW, s, lane, table_row, limit, w);   \
+            process_span<RR, MODE, MASKED, STORE_TABLE>(prev, cur, taps, krange, mask, MW, s, lane, table_row, \
+                                                        limit, w);                                             \
         break;
         SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
         SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
@@ -498,6 +504,25 @@ __device__ __forceinline__ void run_pass(const int cpl, const float *prev, float
 #undef SPDY_CASE
         default: break;
     }
+}
+
+// The finished row goes from shared memory to the walk-back table as ONE bulk copy per layer, issued by one
+// thread and carried out by the copy engine: the table stores then cost the warps no instructions and the
+// load/store data path - the unit this kernel is bound by - no wavefronts.  Both addresses are 16-byte aligned
+// and the size a multiple of 16 bytes (rows start on 128-cell boundaries of a 256-byte aligned table and
+// are whole blocks of 32 cells long).  Protocol per layer: every thread that wrote the row makes its
+// writes visible to the copy engine (bulk_copy_fence), the issuing thread waits until the engine has read
+// the buffer that the next layer will overwrite (bulk_copy_wait_read: that copy was issued a whole layer
+// earlier), the layer's barrier follows, then the issuing thread starts the copy of the row just finished.
+__device__ __forceinline__ void bulk_copy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void bulk_copy_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_copy_row_to_table(void *table_row, const float *row, const int cells)
+{
+    const unsigned src = static_cast<unsigned>(__cvta_generic_to_shared(row));
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(table_row), "r"(src),
+                 "r"(cells * 4)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
 // (value, t) merge with the lowest t among equal values.
@@ -533,7 +558,12 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
 {
     constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
     constexpr int NWARPS = NT / 32;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+#ifdef SPDY_DEBUG_CHECKS
+    constexpr bool BULK = false;  // the debug build stores every table cell itself, index-checked
+#else
+    constexpr bool BULK = ROWFMT && !GROWS;  // rows in shared memory, row-value table: bulk copy per layer
+#endif
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     float *rows;
     int2 *tap_buf;
     if constexpr (GROWS) {
@@ -602,7 +632,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
             // (64 registers per thread: no room to hold the next pass's descriptor across a pass)
             for (int p = p0; p < p1; ++p) {
                 const int2 pd = __ldg(reinterpret_cast<const int2 *>(args.passes + p));
-                run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+                run_pass<MODE, RCAP, false, !BULK>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
                                             args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
             }
         } else {
@@ -611,7 +641,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
             for (int p = p0; p < p1; ++p) {
                 const int2 pd = pd_next;
                 if (p + 1 < p1) pd_next = __ldg(reinterpret_cast<const int2 *>(args.passes + p + 1));
-                run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+                run_pass<MODE, RCAP, false, !BULK>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
                                             args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
             }
         }
@@ -619,13 +649,21 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         // sources); PAD more cells of +inf behind them cover every read of the next layer.
         for (int i = tid; i < PAD; i += NT) cur[ld.extent + i] = INF;
         if (have_next) tap_buf[((l + 1) & 1) * KS + tid] = next_tap;
+        if constexpr (BULK) {
+            bulk_copy_fence();
+            if (tid == 0) bulk_copy_wait_read();
+        }
         __syncthreads();
+        if constexpr (BULK)
+            if (tid == 0) bulk_copy_row_to_table(row_base, cur, ld.extent);
         ld = ld_next;
         p0 = q0;
         p1 = q1;
     }
 
     // min over t <= B of D_L[t], lowest t among equals (the band's upper end never exceeds B).
+    if constexpr (BULK)
+        if (tid == 0) bulk_copy_wait_read();  // the last row's copy must have left shared memory before the CTA does
     const float *last = rows + (L & 1) * args.row_stride + PAD;
     float bv = INF;
     int bt = 0x7fffffff;
@@ -672,7 +710,12 @@ __global__ void __launch_bounds__(kWarpKernelThreads, MINB) spdy_forward_warp_ke
 {
     constexpr bool ROWFMT = (MODE == MODE_ROW || MODE == MODE_ROW2);
     constexpr int NWARPS = kWarpKernelThreads / 32;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+#ifdef SPDY_DEBUG_CHECKS
+    constexpr bool BULK = false;
+#else
+    constexpr bool BULK = ROWFMT;  // row-value table: one bulk copy per layer and warp (see bulk_copy_row_to_table)
+#endif
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int64_t n_local = static_cast<int64_t>(blockIdx.x) * NWARPS + warp;
@@ -729,7 +772,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, MINB) spdy_forward_warp_ke
         for (int p = p0; p < p1; ++p) {
             const int2 pd = pd_next;
             if (p + 1 < p1) pd_next = __ldg(reinterpret_cast<const int2 *>(args.passes + p + 1));
-            run_pass<MODE, RCAP, false>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+            run_pass<MODE, RCAP, false, !BULK>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
                                         args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
         }
         for (int i = lane; i < PAD; i += 32) cur[ld.extent + i] = INF;
@@ -737,12 +780,20 @@ __global__ void __launch_bounds__(kWarpKernelThreads, MINB) spdy_forward_warp_ke
             if (lane < ld_next.nslots) tap_buf[((l + 1) & 1) * KS + lane] = next_a;
             if (lane + 32 < ld_next.nslots) tap_buf[((l + 1) & 1) * KS + lane + 32] = next_b;
         }
+        if constexpr (BULK) {
+            bulk_copy_fence();
+            if (lane == 0) bulk_copy_wait_read();
+        }
         __syncwarp();
+        if constexpr (BULK)
+            if (lane == 0) bulk_copy_row_to_table(row_base, cur, ld.extent);
         ld = ld_next;
         p0 = q0;
         p1 = q1;
     }
 
+    if constexpr (BULK)
+        if (lane == 0) bulk_copy_wait_read();
     const float *last = rows + (L & 1) * args.row_stride + PAD;
     float bv = INF;
     int bt = 0x7fffffff;
