@@ -294,6 +294,59 @@ int spdy_uniform_profile(const int32_t *times_host, int32_t L, int32_t K, int32_
                          int32_t *choice_out, int64_t *total_out);
 
 /*
+ * SPDY's search for the sensitivity coefficients (Section 3.3; Appendix B, Algorithm 4) with the dynamic
+ * programs of all pending trials solved as one batch.  Host loop; synchronous.
+ *
+ * Algorithm 4 samples c0 and `trials` more coefficient vectors, keeps the best, then for neighbourhood
+ * sizes d = ceil(delta * L) .. 1 mutates the best vector c* in d random entries `trials` times per size,
+ * accepting a mutation when its profile evaluates strictly better.  What a trial resamples does not depend
+ * on c*, so this call forms the proposals of all remaining trials of a size from the current c* at once,
+ * solves their dynamic programs (Eq. 4 errors, spdy_solve_batch_coeffs_host) as one batch and evaluates
+ * the profiles in trial order up to the first improvement; the proposals behind it are rebuilt from the
+ * new c*.  Decisions, result and the number of evaluations equal the sequential algorithm's.
+ *
+ *   plan         a plan for the timing table and budget (K = plan's K, L = plan's L)
+ *   c0_host      [L] fp32, phase1_host [trials][L] fp32: the random vectors of the first loop (the caller
+ *                draws them: the paper samples uniformly from [0, 1])
+ *   opts         trials (Algorithm 4's k), delta (its neighbourhood fraction), patience: 0 = `trials` trials
+ *                per size as Algorithm 4 prints it, p > 0 = stop a size after p trials in a row without
+ *                improvement, as the text of Section 3.3 says; max_batch: most dynamic programs per solver
+ *                call (0 = 65536)
+ *   draw         called as draw(d, trial, indices[d], values[d], user): the d distinct entries (0 .. L-1) and
+ *                their new values that trial `trial` of size d resamples; must not depend on earlier calls
+ *   eval         eval(profile[L], L, user) -> the loss of that profile (Section 3.4: the calibration loss of
+ *                the stitched model), lower is better; profile bytes 0xFF = infeasible, return +inf
+ *   solve        NULL = this library on the plan's device; else solve(coeffs[n][L], n, profile[n][L], user)
+ *                -> status, which lets the loop run against another solver (tests use the CPU oracle)
+ *   c_out_host [L], profile_out_host [L], *result: the best vector, its profile, loss and counters
+ *   accepted_d_host / accepted_trial_host [accepted_capacity], may be NULL with capacity 0: the accepted
+ *                trials in order, d = 0 for the first loop; result->accepted counts all of them
+ * Errors: INVALID_ARG, NO_MEMORY, NO_DEVICE_CODE (solve NULL on a host-only plan or build), the solver's.
+ */
+typedef double (*spdy_eval_fn)(const uint8_t *profile_host, int32_t L, void *user);
+typedef void (*spdy_draw_fn)(int32_t d, int32_t trial, int32_t *indices_host, float *values_host, void *user);
+typedef int (*spdy_solve_fn)(const float *coeffs_host, int64_t n, uint8_t *profile_host, void *user);
+typedef struct spdy_search_options {
+    int32_t trials;
+    int32_t patience;
+    double delta;
+    int64_t max_batch;
+} spdy_search_options;
+typedef struct spdy_search_result {
+    double loss;
+    int64_t evals;         /* calls of eval */
+    int64_t accepted;      /* accepted trials */
+    int64_t dp_batches;    /* solver calls */
+    int64_t dp_candidates; /* dynamic programs solved */
+    double dp_seconds, eval_seconds;
+} spdy_search_result;
+int spdy_search(spdy_plan *plan, const float *c0_host, const float *phase1_host, const spdy_search_options *opts,
+                spdy_draw_fn draw, void *draw_user, spdy_eval_fn eval, void *eval_user, spdy_solve_fn solve,
+                void *solve_user, void *cuda_stream, float *c_out_host, uint8_t *profile_out_host,
+                spdy_search_result *result, int32_t *accepted_d_host, int32_t *accepted_trial_host,
+                int64_t accepted_capacity);
+
+/*
  * One-shot form of the whole path, in the shape of the problem statement of Section 3.1 (Eq. 1: errors
  * e_l^s, times t_l^s, budget T in, one choice per layer out): errors[N][L][K], times[L][K], budget B ->
  * profile, cost, time_used, all device pointers on the current device.  Reads times back to

@@ -29,12 +29,12 @@ EXPORTS = (
     "spdy_solve_batch_coeffs", "spdy_solve_batch_coeffs_host", "spdy_quadratic_errors",
     "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile", "spdy_probe_peaks",
     "spdy_plan_get_tables", "spdy_plan_verify", "spdy_plan_status_word", "spdy_debug_checks_enabled",
-    "spdy_plan_shape_for_batch",
+    "spdy_plan_shape_for_batch", "spdy_search",
 )
 # What the host-only library holds (everything that needs no CUDA).
 HOST_EXPORTS = (
     "spdy_plan_create", "spdy_plan_destroy", "spdy_plan_get_info", "spdy_plan_get_bands", "spdy_workspace_bytes",
-    "spdy_plan_get_tables", "spdy_plan_verify", "spdy_plan_shape_for_batch", "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile",
+    "spdy_plan_get_tables", "spdy_plan_verify", "spdy_plan_shape_for_batch", "spdy_search", "spdy_time_target", "spdy_bucketize_times", "spdy_uniform_profile",
     "spdy_strerror", "spdy_version",
 )
 
@@ -44,6 +44,24 @@ class SpdyOptions(ctypes.Structure):
                 ("cluster", ctypes.c_int32), ("forward_mode", ctypes.c_int32),
                 ("rows_in_global", ctypes.c_int32), ("kernel", ctypes.c_int32),
                 ("schedule", ctypes.c_int32), ("auto_shape", ctypes.c_int32)]
+
+
+class SpdySearchOptions(ctypes.Structure):
+    _fields_ = [("trials", ctypes.c_int32), ("patience", ctypes.c_int32), ("delta", ctypes.c_double),
+                ("max_batch", ctypes.c_int64)]
+
+
+class SpdySearchResult(ctypes.Structure):
+    _fields_ = [("loss", ctypes.c_double), ("evals", ctypes.c_int64), ("accepted", ctypes.c_int64),
+                ("dp_batches", ctypes.c_int64), ("dp_candidates", ctypes.c_int64),
+                ("dp_seconds", ctypes.c_double), ("eval_seconds", ctypes.c_double)]
+
+
+EVAL_FN = ctypes.CFUNCTYPE(ctypes.c_double, ctypes.POINTER(ctypes.c_uint8), ctypes.c_int32, ctypes.c_void_p)
+DRAW_FN = ctypes.CFUNCTYPE(None, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32),
+                           ctypes.POINTER(ctypes.c_float), ctypes.c_void_p)
+SOLVE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.c_int64,
+                            ctypes.POINTER(ctypes.c_uint8), ctypes.c_void_p)
 
 
 class SpdyPlanTables(ctypes.Structure):
@@ -106,6 +124,9 @@ def _configure(lib, host_only: bool = False):
     lib.spdy_plan_shape_for_batch.argtypes = [vp, i64, ctypes.c_size_t]
     lib.spdy_workspace_bytes.restype = ctypes.c_size_t
     lib.spdy_workspace_bytes.argtypes = [vp, i64]
+    lib.spdy_search.restype = ctypes.c_int
+    lib.spdy_search.argtypes = [vp, vp, vp, ctypes.POINTER(SpdySearchOptions), DRAW_FN, vp, EVAL_FN, vp, SOLVE_FN, vp,
+                                vp, vp, vp, ctypes.POINTER(SpdySearchResult), vp, vp, i64]
     lib.spdy_time_target.restype = ctypes.c_double
     lib.spdy_time_target.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double]
     lib.spdy_bucketize_times.restype = ctypes.c_int

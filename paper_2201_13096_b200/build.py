@@ -5,8 +5,8 @@ Three shared objects come out of ``csrc/``:
 * ``libspdy_dp.so``        - the product: host plan (g++) + kernels and launch code (nvcc);
 * ``libspdy_dp_debug.so``  - the same sources with ``-DSPDY_DEBUG_CHECKS``: every row and table access of
   the forward kernels checks its index and reports through the plan's status word (for tests);
-* ``libspdy_plan_host.so`` - ``spdy_plan.cpp`` alone, built with the host compiler: plans, their
-  verification and the host helpers, for machines and tests without nvcc.
+* ``libspdy_plan_host.so`` - ``spdy_plan.cpp`` and ``spdy_search.cpp`` alone, built with the host compiler:
+  plans, their verification, the host helpers and the search loop, for machines and tests without nvcc.
 
 Translation units compile in parallel and only when they or a header changed.
 """
@@ -22,7 +22,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 HEADERS = [os.path.join(os.path.dirname(PKG), "include", "spdy_dp.h"),
            os.path.join(CSRC, "spdy_plan.h"), os.path.join(CSRC, "spdy_device.cuh")]
-HOST_SOURCE = os.path.join(CSRC, "spdy_plan.cpp")
+HOST_SOURCES = [os.path.join(CSRC, "spdy_plan.cpp"), os.path.join(CSRC, "spdy_search.cpp")]
 LIB = os.path.join(PKG, "libspdy_dp.so")
 LIB_DEBUG = os.path.join(PKG, "libspdy_dp_debug.so")
 LIB_HOST = os.path.join(PKG, "libspdy_plan_host.so")
@@ -65,9 +65,9 @@ def _run(cmd, log=None):
 
 def build_host(force: bool = False) -> str:
     """``libspdy_plan_host.so``: the host side alone, host compiler only."""
-    if force or _stale(LIB_HOST, [HOST_SOURCE, HEADERS[0], HEADERS[1]]):
+    if force or _stale(LIB_HOST, HOST_SOURCES + [HEADERS[0], HEADERS[1]]):
         tmp = LIB_HOST + f".tmp{os.getpid()}"
-        _run(["g++", *GXX_FLAGS, "-shared", "-o", tmp, HOST_SOURCE])
+        _run(["g++", *GXX_FLAGS, "-shared", "-o", tmp, *HOST_SOURCES])
         os.replace(tmp, LIB_HOST)
     return LIB_HOST
 
@@ -78,7 +78,7 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     to stdout."""
     lib = LIB_DEBUG if debug else LIB
     sources = cuda_sources()
-    if not force and not _stale(lib, sources + [HOST_SOURCE] + HEADERS):
+    if not force and not _stale(lib, sources + HOST_SOURCES + HEADERS):
         return lib
     objdir = os.path.join(OBJ_ROOT, "debug" if debug else "release")
     os.makedirs(objdir, exist_ok=True)
@@ -89,10 +89,11 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
         objects.append(obj)
         if force or verbose or _stale(obj, [src] + HEADERS):
             jobs.append([_nvcc(), *NVCC_FLAGS, *defines, *(["-Xptxas", "-v"] if verbose else []), "-c", "-o", obj, src])
-    host_obj = os.path.join(objdir, "spdy_plan.cpp.o")
-    objects.append(host_obj)
-    if force or _stale(host_obj, [HOST_SOURCE, HEADERS[0], HEADERS[1]]):
-        jobs.append(["g++", *GXX_FLAGS, *defines, "-c", "-o", host_obj, HOST_SOURCE])
+    for src in HOST_SOURCES:
+        host_obj = os.path.join(objdir, os.path.basename(src) + ".o")
+        objects.append(host_obj)
+        if force or _stale(host_obj, [src, HEADERS[0], HEADERS[1]]):
+            jobs.append(["g++", *GXX_FLAGS, *defines, "-c", "-o", host_obj, src])
     with ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 1))) as pool:
         list(pool.map(lambda cmd: _run(cmd, log), jobs))
     tmp = lib + f".tmp{os.getpid()}"

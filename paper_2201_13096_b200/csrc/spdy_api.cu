@@ -476,7 +476,9 @@ int hook_attach(spdy_plan *p)
     return rc;
 }
 
-const DeviceHooks kHooks = {hook_limits, hook_attach, hook_release};
+int hook_solve_coeffs_host(spdy_plan *p, const float *coeffs_host, int64_t n, uint8_t *profile_host, void *cuda_stream);
+
+const DeviceHooks kHooks = {hook_limits, hook_attach, hook_release, hook_solve_coeffs_host};
 
 struct HookRegistration {
     HookRegistration() { register_device_hooks(&kHooks); }
@@ -785,6 +787,22 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
     }
     SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
     return SPDY_OK;
+}
+
+// The search's solver: coefficients up, profiles down, self-check word read.
+int hook_solve_coeffs_host(spdy_plan *p, const float *coeffs_host, int64_t n, uint8_t *profile_host, void *cuda_stream)
+{
+    std::vector<float> cost;
+    std::vector<int32_t> time_used;
+    try {
+        cost.resize(static_cast<size_t>(n));
+        time_used.resize(static_cast<size_t>(n));
+    } catch (const std::bad_alloc &) {
+        return SPDY_ERR_NO_MEMORY;
+    }
+    int rc = solve_host_impl(p, coeffs_host, true, n, profile_host, cost.data(), time_used.data(), cuda_stream);
+    if (rc == SPDY_OK) rc = spdy_plan_check_status(p, cuda_stream);
+    return rc;
 }
 
 }  // namespace

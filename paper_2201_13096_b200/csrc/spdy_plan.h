@@ -208,6 +208,8 @@ struct DeviceHooks {
     int (*limits)(int device, DeviceLimits *out);
     int (*attach)(spdy_plan *p);    // set kernel attributes, verify occupancy, upload the tables
     void (*release)(spdy_plan *p);  // free everything behind p->dev
+    // Eq. 4 coefficients [n][L] in host memory -> profiles [n][L] in host memory (the search's solver)
+    int (*solve_coeffs_host)(spdy_plan *p, const float *coeffs_host, int64_t n, uint8_t *profile_host, void *cuda_stream);
 };
 void register_device_hooks(const DeviceHooks *hooks);
 const DeviceHooks *device_hooks();

@@ -50,6 +50,34 @@ def test_host_logic_of_the_batched_search(seed, patience):
     same_result(small, ref)
 
 
+def test_search_entry_point_checks_its_arguments_and_passes_failures_on():
+    import ctypes
+
+    from paper_2201_13096_b200 import binding
+
+    wl, loss, c0, phase1, draws = problem(3, 4)
+    solver = oracle_solver(wl.times, wl.B)
+    with pytest.raises(ZeroDivisionError):  # an exception inside a callback comes back out of the call
+        S.search(wl.times, wl.B, c0, phase1, draws, lambda p: 1 / 0, trials=4, solver=solver)
+    with pytest.raises(ValueError):  # so does the failure of a solver callback (here: profiles of the wrong shape)
+        S.search(wl.times, wl.B, c0, phase1, draws, loss, trials=4, solver=lambda c: np.zeros((1, 1)))
+    lib = binding.library()
+    plan = binding.Plan(wl.times, wl.B, device=-1)
+    res = binding.SpdySearchResult()
+    opts = binding.SpdySearchOptions(trials=4, patience=0, delta=0.3, max_batch=0)
+    out_c, out_p = np.empty(wl.L, np.float32), np.empty(wl.L, np.uint8)
+    vp = ctypes.c_void_p
+    args = [plan._h, c0.ctypes.data_as(vp), phase1.ctypes.data_as(vp), ctypes.byref(opts), binding.DRAW_FN(lambda *a: None),
+            None, binding.EVAL_FN(lambda *a: 0.0), None, binding.SOLVE_FN(0), None, None, out_c.ctypes.data_as(vp),
+            out_p.ctypes.data_as(vp), ctypes.byref(res), None, None, 0]
+    assert lib.spdy_search(*args) == -8  # no solver given and the plan has no device
+    bad = list(args)
+    bad[0] = None
+    assert lib.spdy_search(*bad) == -1
+    opts.delta = 1.5
+    assert lib.spdy_search(*args) == -1
+
+
 def test_special_cases_of_the_batched_search():
     wl, loss, c0, phase1, draws = problem(21, 6)
     solver = oracle_solver(wl.times, wl.B)
