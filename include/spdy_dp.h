@@ -100,7 +100,7 @@ typedef struct spdy_options {
                               wasted on slots that overlap a pass only partly); 3 = passes sized by dynamic
                               programming and dealt to the warps by load (least waste, most passes, measured
                               slowest; for measurement).  Bits 8-15: upper limit of cells per lane per pass,
-                              1..24 (0 = the kernel's own limit; for measurement) */
+                              1..48 (0 = the kernel's own limit; for measurement) */
     int32_t auto_shape;    /* 0: when threads, cluster, rows_in_global and kernel are all 0 the plan also lays
                               out launch shapes for batches too small to fill the device (larger CTAs, clusters
                               of 2/4/8) and spdy_solve_batch picks by N; 1: never, one shape for every N */

@@ -493,7 +493,7 @@ __device__ __forceinline__ void run_pass(const int cpl, const float *prev, float
     switch (cpl) {
 #define SPDY_CASE(RR)                                                                                          \
     case RR:                                                                                                   \
-        if constexpr (RR <= kRmax && RR <= RCAP)                                                               \
+        if constexpr (RR <= kRmaxLong && RR <= RCAP)                                                           \
             process_span<RR, MODE, MASKED, STORE_TABLE>(prev, cur, taps, krange, mask, MW, s, lane, table_row, \
                                                         limit, w);                                             \
         break;
@@ -501,6 +501,8 @@ __device__ __forceinline__ void run_pass(const int cpl, const float *prev, float
         SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
         SPDY_CASE(13) SPDY_CASE(14) SPDY_CASE(15) SPDY_CASE(16) SPDY_CASE(17) SPDY_CASE(18)
         SPDY_CASE(19) SPDY_CASE(20) SPDY_CASE(21) SPDY_CASE(22) SPDY_CASE(23) SPDY_CASE(24)
+        SPDY_CASE(25) SPDY_CASE(26) SPDY_CASE(27) SPDY_CASE(28) SPDY_CASE(29) SPDY_CASE(30) SPDY_CASE(31) SPDY_CASE(32) SPDY_CASE(33) SPDY_CASE(34) SPDY_CASE(35) SPDY_CASE(36)
+        SPDY_CASE(37) SPDY_CASE(38) SPDY_CASE(39) SPDY_CASE(40) SPDY_CASE(41) SPDY_CASE(42) SPDY_CASE(43) SPDY_CASE(44) SPDY_CASE(45) SPDY_CASE(46) SPDY_CASE(47) SPDY_CASE(48)
 #undef SPDY_CASE
         default: break;
     }
@@ -1032,8 +1034,8 @@ VariantList variants_row2();
 // a 1024-thread CTA (64 registers per thread) can unroll without spilling.
 template <int MODE> constexpr int ctas_256() { return MODE == MODE_ARG_PAIR ? 2 : 3; }
 #define SPDY_CTA_VARIANTS(MODE)                                                                                 \
-    SPDY_CTA_VARIANT(MODE, 128, 4, kRmax), SPDY_CTA_VARIANT(MODE, 256, ctas_256<MODE>(), kRmax),                  \
-    SPDY_CTA_VARIANT(MODE, 512, 1, kRmax), SPDY_CTA_VARIANT(MODE, 1024, 1, cells_per_lane_1024(MODE)),          \
+    SPDY_CTA_VARIANT(MODE, 128, 4, long_pass_cap(MODE)), SPDY_CTA_VARIANT(MODE, 256, ctas_256<MODE>(), kRmax),    \
+    SPDY_CTA_VARIANT(MODE, 512, 1, long_pass_cap(MODE)), SPDY_CTA_VARIANT(MODE, 1024, 1, cells_per_lane_1024(MODE)), \
     SPDY_CTA_VARIANT(MODE, 128, 6, 8), SPDY_CTA_VARIANT(MODE, 256, 3, 8),                                       \
     SPDY_CTA_VARIANT(MODE, 512, 1, 8), SPDY_CTA_VARIANT(MODE, 1024, 1, 8)
 #define SPDY_FULL_VARIANTS(MODE)                                                                                \
@@ -1042,9 +1044,8 @@ template <int MODE> constexpr int ctas_256() { return MODE == MODE_ARG_PAIR ? 2 
                spdy_forward_kernel<MODE, 1024, 1, global_rows_cap_1024(MODE), true>},                           \
     FwdVariant{KERNEL_CTA_GLOBAL, MODE, 512, kRmax, spdy_forward_kernel<MODE, 512, 1, kRmax, true>},            \
     FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, 8, spdy_forward_warp_kernel<MODE, 8, 8>},                 \
-    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, warp_mid_cap(MODE),                                       \
-               spdy_forward_warp_kernel<MODE, 6, warp_mid_cap(MODE)>},                                          \
-    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, kRmax, spdy_forward_warp_kernel<MODE, 4, kRmax>}
+    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, long_pass_cap(MODE),                                      \
+               spdy_forward_warp_kernel<MODE, 4, long_pass_cap(MODE)>}
 #define SPDY_CLUSTER_VARIANTS(MODE) \
     ClusterVariant{MODE, 256, spdy_forward_cluster_kernel<MODE, 256>}, ClusterVariant{MODE, 512, spdy_forward_cluster_kernel<MODE, 512>}
 

@@ -154,7 +154,8 @@ void build_slots(spdy_plan *p, int merge)
 int cells_per_lane_cap(int kind, int threads, int mode)
 {
     if (kind == KERNEL_CTA_GLOBAL) return threads >= 1024 ? global_rows_cap_1024(mode) : kRmax;
-    if (kind == KERNEL_WARP) return kRmax;
+    if (kind == KERNEL_WARP) return long_pass_cap(mode);
+    if (threads == 128 || threads == 512) return long_pass_cap(mode);  // 128 registers per thread available
     return threads >= 1024 ? cells_per_lane_1024(mode) : kRmax;
 }
 
@@ -162,7 +163,7 @@ int cells_per_lane_cap(int kind, int threads, int mode)
 int rcap_for(int kind, int threads, int mode, int max_cpl)
 {
     if (kind == KERNEL_CTA_GLOBAL) return cells_per_lane_cap(kind, threads, mode);
-    if (kind == KERNEL_WARP) return max_cpl <= 8 ? 8 : (max_cpl <= warp_mid_cap(mode) ? warp_mid_cap(mode) : kRmax);
+    if (kind == KERNEL_WARP) return max_cpl <= 8 ? 8 : long_pass_cap(mode);
     return max_cpl <= 8 ? 8 : cells_per_lane_cap(kind, threads, mode);
 }
 
@@ -215,11 +216,11 @@ void plan_layer_passes(const std::vector<int> &ba, const std::vector<int> &bb, i
     }
     auto overlapping = [&](int i, int j) { return started[std::min(j, nb + 1)] - ended[std::min(i, nb + 1)]; };
     // Cost of a pass in wavefronts of the shared-memory data path, the unit the kernel is bound by: one per
-    // slot and 32 cells, the 16-byte slot-pair reads (two wavefronts per pair), the stores of the new row
-    // (shared memory and table), and the pass's own descriptor and set-up.
+    // slot and 32 cells, the 16-byte slot-pair reads (measured: about three wavefronts per pair), the stores
+    // of the new row, and the pass's own descriptor and set-up.
     auto pass_cost = [&](int i, int j) {
         const int n = overlapping(i, j);
-        return static_cast<double>(n) * ((j - i) + 1.0) + 2.3 * (j - i) + 6.0;
+        return static_cast<double>(n) * ((j - i) + 1.5) + 1.3 * (j - i) + 6.0;
     };
     auto finish = [&](std::vector<PassPlan> &passes) {
         for (PassPlan &pp : passes) {
@@ -577,29 +578,22 @@ bool warp_kernel_fits(const spdy_plan *p)
                                 : (max_slots <= 64 && p->mode == MODE_ARG_PAIR);
 }
 
-// The warp kernel's builds unroll passes of up to 24, warp_mid_cap() or 8 cells per lane in 128, 80 and 64
-// registers per thread, which lets 4, 6 and 8 CTAs of 128 threads share an SM.  Longer passes are cheaper
-// per cell, but only while registers do not cost resident warps that shared memory would allow: take the
-// longest pass whose register limit is no tighter than the shared-memory limit.
+// The warp kernel's two builds unroll passes of up to 8 cells per lane in 64 registers (8 CTAs of 128
+// threads per SM) or up to long_pass_cap() in 128 registers (4 CTAs).  Measured over budgets of 750 to 3000
+// buckets: while shared memory lets seven or more CTAs share an SM the short passes with twice the resident
+// warps win (B = 1000: 0.53 against 0.62 ms); from there on one long pass per layer does (B = 1500: 0.73
+// against 0.99 ms).
 int choose_warp_shape(spdy_plan *p)
 {
     const int threads = 128;
     const int asked_cap = p->pass_cap;
     int rc = layout_table(p, KERNEL_WARP, threads, nullptr);
     if (rc != SPDY_OK) return rc;
-    if (asked_cap == 0) {
-        const int by_smem = std::min(8, resident_ctas(p, threads, p->smem_bytes));
-        const int caps[3] = {kRmax, warp_mid_cap(p->mode), 8}, by_regs[3] = {4, 6, 8};
-        for (int i = 0; i < 3; ++i)
-            if (by_regs[i] >= by_smem || i == 2) {
-                if (caps[i] < p->rcap) {
-                    p->pass_cap = caps[i];
-                    rc = layout_table(p, KERNEL_WARP, threads, nullptr);
-                    p->pass_cap = asked_cap;
-                    if (rc != SPDY_OK) return rc;
-                }
-                break;
-            }
+    if (asked_cap == 0 && p->rcap > 8 && resident_ctas(p, threads, p->smem_bytes) >= 7) {
+        p->pass_cap = 8;
+        rc = layout_table(p, KERNEL_WARP, threads, nullptr);
+        p->pass_cap = asked_cap;
+        if (rc != SPDY_OK) return rc;
     }
     if (p->smem_bytes > p->limits.smem_per_block - kStaticSmemReserve) return SPDY_ERR_UNSUPPORTED;
     p->kind = KERNEL_WARP;
@@ -622,7 +616,7 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
     }
     p->schedule = opts ? (opts->schedule & 0xFF) : 0;
     p->pass_cap = opts ? ((opts->schedule >> 8) & 0xFF) : 0;
-    if (p->schedule < 0 || p->schedule > SCHED_SIZED || (opts && (opts->schedule >> 16) != 0) || p->pass_cap > kRmax)
+    if (p->schedule < 0 || p->schedule > SCHED_SIZED || (opts && (opts->schedule >> 16) != 0) || p->pass_cap > kRmaxLong)
         return SPDY_ERR_INVALID_ARG;
     // Left open: levelled passes where the shared-memory data path binds (row-value table); passes of one
     // length where instruction issue binds (byte table: one unrolled body per layer measured 3 % faster).

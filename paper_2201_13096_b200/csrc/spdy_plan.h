@@ -14,10 +14,17 @@
 
 namespace spdy {
 
-constexpr int kLibraryVersion = 2002;
+constexpr int kLibraryVersion = 2003;
 
 // Most band cells one lane owns in one warp pass; the kernels unroll passes of 1..kRmax cells per lane.
 constexpr int kRmax = 24;
+
+// The builds with 128 registers per thread to themselves (128-thread CTAs at four per SM) and the cheapest
+// cell update (packed add + 3-input minimum) unroll passes twice as long: every pass pays for its own
+// 16-byte slot reads (about three data-path wavefronts per pair of slots), so half as many passes take
+// 4 % off the traffic of the unit the kernel is bound by.
+constexpr int kRmaxLong = 48;
+constexpr int long_pass_cap(int mode) { return mode == 4 /* MODE_ROW2 */ ? kRmaxLong : kRmax; }
 
 // Widest band (cells) for which the plan considers one warp per candidate when left to choose (it then
 // takes it if at least three CTAs of four candidates fit an SM).
@@ -44,10 +51,8 @@ constexpr int cluster_cells_per_lane(int threads) { return threads >= 512 ? 16 :
 // row addresses).
 constexpr int global_rows_cap_1024(int mode) { return mode == MODE_ARG_PAIR ? 8 : 12; }
 
-// The warp-per-candidate kernel comes in three builds: passes of up to 8 cells per lane in 64 registers
-// (8 CTAs of 128 threads per SM), up to warp_mid_cap() in 80 registers (6 CTAs), up to kRmax in 128 (4 CTAs).
-constexpr int warp_mid_cap(int mode) { return mode == MODE_ARG_PAIR ? 12 : 18; }
-
+// The warp-per-candidate kernel comes in two builds: passes of up to 8 cells per lane in 64 registers
+// (8 CTAs of 128 threads per SM) and up to long_pass_cap() in 128 registers (4 CTAs).
 inline bool mode_is_row(int mode) { return mode == MODE_ROW || mode == MODE_ROW2; }
 inline bool mode_is_arg(int mode) { return mode == MODE_ARG || mode == MODE_ARG_PRED || mode == MODE_ARG_PAIR; }
 

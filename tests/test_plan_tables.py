@@ -250,8 +250,10 @@ def test_pass_schedules_trade_wasted_updates_against_passes():
     assert d <= info[3]["issued_updates"] < info[2]["issued_updates"] < info[1]["issued_updates"] < 1.06 * d
     assert info[0]["issued_updates"] == info[2]["issued_updates"] < 1.03 * d
     assert passes[2] <= 1.05 * passes[1] and passes[3] > 1.2 * passes[1]
-    u8 = binding.Plan(wl.times, wl.B, device=-1, auto_shape=1, table_format=U8).info
-    assert u8["issued_updates"] == info[1]["issued_updates"]  # the byte table keeps passes of one length
+    u8 = {s: binding.Plan(wl.times, wl.B, device=-1, auto_shape=1, table_format=U8, schedule=s).info for s in (0, 1)}
+    assert u8[0]["issued_updates"] == u8[1]["issued_updates"]  # the byte table keeps passes of one length
+    # the fp32 table's 128-thread build unrolls passes twice as long: half as many passes
+    assert passes[1] < 0.6 * binding.Plan(wl.times, wl.B, device=-1, auto_shape=1, table_format=U8, schedule=1).tables(0)["n_passes"]
 
 
 def test_small_batches_get_their_own_launch_shapes():
