@@ -168,7 +168,8 @@ int spdy_plan_get_bands(const spdy_plan *plan, int32_t *lo_host, int32_t *width_
  * if there is none), i >= 1 = the i-th launch shape for small batches.  The pointers stay valid until the
  * plan is destroyed.
  *   layers      [L][8] int32: width, row offset in the table, lo, smallest usable time, extent (cells the
- *               passes write, a multiple of 32), shift slots, 0, 0
+ *               passes write, a multiple of 32), shift slots, fill (cells of +inf refilled behind the row:
+ *               as far as the next layer reads beyond the extent), 0
  *   slots       [L][K][2] int32: (a, b) of each shift slot: it contributes to band cells a..b and reads the
  *               previous row at cell - a (the first layers[l][5] entries of a layer are valid)
  *   passes      [n_passes][2]: first cell, and u_lo | u_hi << 8 | dense << 16 | cells_per_lane << 24
@@ -188,7 +189,7 @@ typedef struct spdy_plan_tables {
     int32_t kernel_kind;         /* 0 CTA per candidate, 1 CTA with rows in global memory, 2 cluster, 3 warp per candidate */
     int32_t threads, warps_per_candidate, cluster, forward_mode;
     int32_t max_cells_per_lane;  /* the kernel build's largest pass */
-    int32_t row_stride, pad;     /* floats per row buffer; guard cells of +inf on either side of a row */
+    int32_t row_stride, pad;     /* floats per row buffer; guard cells of +inf below cell 0 of a row */
     int32_t out_stride, win_stride; /* cluster shape: floats per slice buffer and per window */
     int32_t mask_words, n_passes;
     int64_t pitch;               /* table cells per candidate */

@@ -50,7 +50,7 @@ struct FwdArgs {
     int64_t n_count;          // candidates of this wave
     int32_t L, K;
     int32_t row_stride;       // floats per row buffer
-    int32_t pad;              // +inf guard cells on either side of a row
+    int32_t pad;              // +inf guard cells below cell 0 of a row
     float *grows;             // row buffers in global memory (GROWS kernels), else null
     int64_t grows_stride;     // floats between the row buffers of consecutive candidates
     const uint8_t *cand_flags; // per candidate of the wave, or null: run only candidates whose flag == which
@@ -623,7 +623,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
         AccessWindow w;
 #ifdef SPDY_DEBUG_CHECKS
         w.read_lo = -PAD;
-        w.read_hi = l == 0 ? args.row_stride - PAD : args.layers[l - 1].extent + PAD;
+        w.read_hi = l == 0 ? args.row_stride - PAD : args.layers[l - 1].extent + args.layers[l - 1].fill;
         w.write_hi = ld.extent;
         w.table_hi = args.pitch - ld.rowoff;
         w.status = args.status;
@@ -648,8 +648,8 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
             }
         }
         // Cells [width, extent) of the new row were written as +inf by the passes (they saw only +inf
-        // sources); PAD more cells of +inf behind them cover every read of the next layer.
-        for (int i = tid; i < PAD; i += NT) cur[ld.extent + i] = INF;
+        // sources); `fill` more cells of +inf behind them cover every read of the next layer.
+        for (int i = tid; i < ld.fill; i += NT) cur[ld.extent + i] = INF;
         if (have_next) tap_buf[((l + 1) & 1) * KS + tid] = next_tap;
         if constexpr (BULK) {
             bulk_copy_fence();
@@ -762,7 +762,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, MINB) spdy_forward_warp_ke
         AccessWindow w;
 #ifdef SPDY_DEBUG_CHECKS
         w.read_lo = -PAD;
-        w.read_hi = l == 0 ? args.row_stride - PAD : args.layers[l - 1].extent + PAD;
+        w.read_hi = l == 0 ? args.row_stride - PAD : args.layers[l - 1].extent + args.layers[l - 1].fill;
         w.write_hi = ld.extent;
         w.table_hi = args.pitch - ld.rowoff;
         w.status = args.status;
@@ -777,7 +777,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, MINB) spdy_forward_warp_ke
             run_pass<MODE, RCAP, false, !BULK>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
                                         args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
         }
-        for (int i = lane; i < PAD; i += 32) cur[ld.extent + i] = INF;
+        for (int i = lane; i < ld.fill; i += 32) cur[ld.extent + i] = INF;
         if (l + 1 < L) {
             if (lane < ld_next.nslots) tap_buf[((l + 1) & 1) * KS + lane] = next_a;
             if (lane + 32 < ld_next.nslots) tap_buf[((l + 1) & 1) * KS + lane + 32] = next_b;

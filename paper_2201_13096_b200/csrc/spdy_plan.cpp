@@ -362,7 +362,8 @@ int layout_table(spdy_plan *p, int kind, int threads, double *efficiency)
     p->pass_masks.clear();
     p->pass_ptr.assign(static_cast<size_t>(p->L) * W + 1, 0);
     int64_t off = 0, max_extent = 32, max_cpl = 1;
-    int64_t need_left = 0, need_right = 0;
+    int64_t need_left = 0;
+    std::vector<int64_t> need_right(static_cast<size_t>(p->L) + 1, 0);  // cells beyond row l-1's extent that layer l reads
     double sum_cost = 0.0, sum_span = 0.0;
     p->issued_updates = 0;
     std::vector<int> ba, bb;
@@ -407,8 +408,7 @@ int layout_table(spdy_plan *p, int kind, int threads, double *efficiency)
                         p->issued_updates += cells;
                         // Lowest and highest previous-row cell a lane of this pass reads through this slot.
                         need_left = std::max<int64_t>(need_left, tr.a - start);
-                        const int64_t prev_e = l == 0 ? 0 : prev_extent;
-                        need_right = std::max<int64_t>(need_right, (start + cells - 1 - tr.a) - (prev_e - 1));
+                        if (l > 0) need_right[l] = std::max<int64_t>(need_right[l], (start + cells - 1 - tr.a) - (prev_extent - 1));
                     }
                 }
                 const uint32_t dense = (count == u_hi - u_lo) ? 1u : 0u;
@@ -423,17 +423,29 @@ int layout_table(spdy_plan *p, int kind, int threads, double *efficiency)
     p->pass_ptr[static_cast<size_t>(p->L) * W] = static_cast<int32_t>(p->passes.size());
     p->pitch = off;
     // Guard cells of +inf on either side of a row: reads of a pass that only partly overlaps a slot's range
-    // land there.  Layer 1 reads the virtual row 0, whose buffer is +inf everywhere but at t = 0, so only the
-    // buffer's end bounds its reads.
-    p->pad = static_cast<int32_t>(std::max<int64_t>(32, round_up(std::max(need_left, need_right), 32)));
-    p->row_stride = static_cast<int32_t>(round_up(max_extent, 32) + 2 * p->pad);
+    // land there.  Below cell 0 the guard is `pad` cells wide (the furthest any pass of the plan reaches) and is
+    // written once; behind a row it is refilled after every layer and only as wide as the NEXT layer reaches
+    // beyond this row's extent (`fill`): bands grow fast while rows are narrow and hardly at all where they
+    // are widest, so the buffer is sized by the largest extent + fill, not by the largest of each.  Layer 1
+    // reads the virtual row 0, whose buffer is +inf everywhere but at t = 0.
+    p->pad = static_cast<int32_t>(std::max<int64_t>(32, round_up(need_left, 32)));
+    int64_t max_row = max_extent;
+    for (int l = 0; l < p->L; ++l) {
+        const int64_t fill = l + 1 < p->L ? round_up(std::max<int64_t>(0, need_right[l + 1]), 32) : 0;
+        p->layers[l].fill = static_cast<int32_t>(fill);
+        max_row = std::max<int64_t>(max_row, p->layers[l].extent + fill);
+    }
+    p->row_stride = static_cast<int32_t>(round_up(max_row, 32) + p->pad);
     p->warps_per_cand = W;
     p->rcap = rcap_for(kind, threads, p->mode, static_cast<int>(max_cpl));
     const int64_t tap_bytes = 2LL * ((K + 1) & ~1) * 8;
     if (kind == KERNEL_CTA_GLOBAL) p->smem_bytes = tap_bytes;
     else if (kind == KERNEL_WARP) p->smem_bytes = (threads / 32) * (2LL * p->row_stride * 4 + tap_bytes);
     else p->smem_bytes = 2LL * p->row_stride * 4 + tap_bytes;
-    if (efficiency) *efficiency = sum_span > 0.0 ? sum_cost / sum_span : 0.0;
+    // Needed cell updates per data-path wavefront the busiest warps take: falls with partly overlapping slots,
+    // with the passes' own slot reads (short passes pay more of them) and with warps that wait for others.
+    (void)sum_cost;
+    if (efficiency) *efficiency = sum_span > 0.0 ? (static_cast<double>(p->distinct_updates) / 32.0) / sum_span : 0.0;
     return SPDY_OK;
 }
 
@@ -799,9 +811,9 @@ int verify_plan(const spdy_plan *p)
     int64_t prev_extent = 0;
     for (int l = 0; l < L; ++l) {
         const LayerDesc &ld = p->layers[l];
-        if (static_cast<int64_t>(ld.extent) + p->pad > buffer_hi) return SPDY_ERR_INTERNAL;  // row and its +inf tail fit
+        if (ld.fill < 0 || static_cast<int64_t>(ld.extent) + ld.fill > buffer_hi) return SPDY_ERR_INTERNAL;  // row and its +inf tail fit
         // Cells of the previous row's buffer known to hold the row or +inf when this layer runs.
-        const int64_t ok_lo = buffer_lo, ok_hi = l == 0 ? buffer_hi : prev_extent + p->pad;
+        const int64_t ok_lo = buffer_lo, ok_hi = l == 0 ? buffer_hi : prev_extent + p->layers[l - 1].fill;
         std::vector<int> covered(ld.extent, 0);
         for (int w = 0; w < W; ++w) {
             const int32_t p0 = p->pass_ptr[static_cast<size_t>(l) * W + w], p1 = p->pass_ptr[static_cast<size_t>(l) * W + w + 1];

@@ -74,7 +74,7 @@ struct LayerDesc {
     int32_t mn;       // smallest usable time of the layer: lo_l = lo_{l-1} + mn
     int32_t extent;   // cells the passes of the layer write (>= width; the excess holds +inf)
     int32_t nslots;   // shift slots of the layer (see TapRange)
-    int32_t reserved0;
+    int32_t fill;     // cells of +inf written behind the row: as far as the next layer reads beyond `extent`
     int32_t reserved1;
 };
 
@@ -150,7 +150,7 @@ struct spdy_plan {
     int pass_cap = 0;        // upper limit of cells per lane per pass asked for by the options (0 = the kernel's)
     spdy::DeviceLimits limits;
     int64_t smem_bytes = 0;
-    int32_t row_stride = 0, pad = 0;  // floats per row buffer; +inf guard cells on either side of a row
+    int32_t row_stride = 0, pad = 0;  // floats per row buffer; +inf guard cells below cell 0 of a row
     // Byte table only: `merged` is a second plan over the same rows and passes whose slots are groups
     // of equal-time choices (ordered by their lowest member); candidates for which that is exact run
     // on it, the others on this plan.  `merge_first` marks such a second plan.

@@ -130,10 +130,13 @@ def test_small_workspace_runs_in_waves(fmt):
     torch.cuda.synchronize()
     assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()),
                 oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES))
-    tiny = torch.empty(plan.workspace_bytes(1) - 256, dtype=torch.uint8, device="cuda")
+    # (a plan with one launch shape: spdy_workspace_bytes of the default plan covers its largest shape)
+    single = binding.Plan(wl.times, wl.B, device=0, table_format=fmt, auto_shape=1)
+    tiny = torch.empty(single.workspace_bytes(1) - 256, dtype=torch.uint8, device="cuda")
     with pytest.raises(binding.SpdyError) as e:
-        binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda(), workspace=tiny)
+        binding.solve_batch(single, torch.from_numpy(wl.errors).cuda(), workspace=tiny)
     assert e.value.status == -2
+    single.close()
     with pytest.raises(binding.SpdyError) as e:  # misaligned workspace
         binding.solve_batch(plan, torch.from_numpy(wl.errors).cuda(), workspace=ws[8:])
     assert e.value.status == -1

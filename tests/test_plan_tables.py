@@ -41,7 +41,7 @@ def check_margins(t):
     """Independent re-derivation of what spdy_plan_verify proves (vectorised over the passes of a layer)."""
     L, K, pad, stride = t["L"], t["K"], t["pad"], t["row_stride"]
     layers, slots, passes = t["layers"], t["slots"].astype(np.int64), t["passes"]
-    width, rowoff, extent, nslots = layers[:, 0], layers[:, 1].astype(np.int64), layers[:, 4], layers[:, 5]
+    width, rowoff, extent, nslots, fill = layers[:, 0], layers[:, 1].astype(np.int64), layers[:, 4], layers[:, 5], layers[:, 6]
     start_all = passes[:, 0].astype(np.int64)
     kr = passes[:, 1].astype(np.uint32)
     u_lo_all, u_hi_all = (kr & 0xFF).astype(int), ((kr >> 8) & 0xFF).astype(int)
@@ -95,12 +95,12 @@ def check_margins(t):
     Wc, ptr = t["warps_per_candidate"], t["pass_ptr"]
     assert len(ptr) == L * Wc + 1 and ptr[-1] == t["n_passes"] and (np.diff(ptr) >= 0).all()
     for l in range(L):
-        assert extent[l] + pad <= stride - pad, "row and its +inf tail must fit the buffer"
+        assert fill[l] >= 0 and extent[l] + fill[l] <= stride - pad, "row and its +inf tail must fit the buffer"
         idx = np.arange(ptr[l * Wc], ptr[(l + 1) * Wc])
         cells = 32 * cpl_all[idx]
         assert (cpl_all[idx] >= 1).all() and (cpl_all[idx] <= t["max_cells_per_lane"]).all()
         assert (start_all[idx] % 32 == 0).all() and (start_all[idx] + cells <= extent[l]).all()
-        check_passes(l, idx, cells, -pad, stride - pad if l == 0 else extent[l - 1] + pad)
+        check_passes(l, idx, cells, -pad, stride - pad if l == 0 else extent[l - 1] + fill[l - 1])
         covered_once(start_all[idx], cells, int(extent[l]))
 
 
@@ -144,7 +144,8 @@ def replay(t, times, errors_one, B, merged):
                     assert not np.isnan(src).any(), "read of a cell nobody wrote"
                     best = np.minimum(best, (src + e[u]).astype(np.float32))
             cur[pad + cells] = best
-        cur[pad + extent:pad + extent + pad] = np.inf
+        cur[pad + extent:pad + extent + int(layers[l, 6])] = np.inf
+        cur[pad + extent + int(layers[l, 6]):] = np.nan  # beyond the refilled tail nothing may be read
     last = buf[L & 1][pad:pad + int(layers[L - 1, 0])]
     if not np.isfinite(last).any():
         return np.float32(np.inf), -1
