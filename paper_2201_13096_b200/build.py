@@ -104,8 +104,31 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     return lib
 
 
+def spilling_kernels(log: str) -> list:
+    """Kernels that ptxas reports with register spills in a ``-Xptxas -v`` log."""
+    import re
+
+    bad = []
+    for name, stores in re.findall(r"Function properties for (\S+)\n\s+\d+ bytes stack frame, (\d+) bytes spill stores", log):
+        if int(stores) > 0:
+            bad.append(name)
+    return bad
+
+
 def build_all(force: bool = False) -> None:
-    build(force=force)
+    """All three libraries; a forced build also checks that no kernel of the product library spills."""
+    if force:
+        import contextlib
+        import io
+
+        buf = io.StringIO()
+        with contextlib.redirect_stdout(buf):
+            build(force=True, verbose=True)
+        bad = spilling_kernels(buf.getvalue())
+        if bad:
+            raise RuntimeError("kernels with register spills: " + ", ".join(bad))
+    else:
+        build()
     build(force=force, debug=True)
     build_host(force=force)
 

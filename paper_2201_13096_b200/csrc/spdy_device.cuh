@@ -1043,7 +1043,8 @@ template <int MODE> constexpr int ctas_256() { return MODE == MODE_ARG_PAIR ? 2 
     FwdVariant{KERNEL_CTA_GLOBAL, MODE, 1024, global_rows_cap_1024(MODE),                                       \
                spdy_forward_kernel<MODE, 1024, 1, global_rows_cap_1024(MODE), true>},                           \
     FwdVariant{KERNEL_CTA_GLOBAL, MODE, 512, kRmax, spdy_forward_kernel<MODE, 512, 1, kRmax, true>},            \
-    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, 8, spdy_forward_warp_kernel<MODE, 8, 8>},                 \
+    FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, warp_short_cap(MODE),                                     \
+               spdy_forward_warp_kernel<MODE, 8, warp_short_cap(MODE)>},                                        \
     FwdVariant{KERNEL_WARP, MODE, kWarpKernelThreads, long_pass_cap(MODE),                                      \
                spdy_forward_warp_kernel<MODE, 4, long_pass_cap(MODE)>}
 #define SPDY_CLUSTER_VARIANTS(MODE) \

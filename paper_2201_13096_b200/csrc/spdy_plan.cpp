@@ -163,7 +163,7 @@ int cells_per_lane_cap(int kind, int threads, int mode)
 int rcap_for(int kind, int threads, int mode, int max_cpl)
 {
     if (kind == KERNEL_CTA_GLOBAL) return cells_per_lane_cap(kind, threads, mode);
-    if (kind == KERNEL_WARP) return max_cpl <= 8 ? 8 : long_pass_cap(mode);
+    if (kind == KERNEL_WARP) return max_cpl <= warp_short_cap(mode) ? warp_short_cap(mode) : long_pass_cap(mode);
     return max_cpl <= 8 ? 8 : cells_per_lane_cap(kind, threads, mode);
 }
 
@@ -601,8 +601,8 @@ int choose_warp_shape(spdy_plan *p)
     const int asked_cap = p->pass_cap;
     int rc = layout_table(p, KERNEL_WARP, threads, nullptr);
     if (rc != SPDY_OK) return rc;
-    if (asked_cap == 0 && p->rcap > 8 && resident_ctas(p, threads, p->smem_bytes) >= 7) {
-        p->pass_cap = 8;
+    if (asked_cap == 0 && p->rcap > warp_short_cap(p->mode) && resident_ctas(p, threads, p->smem_bytes) >= 7) {
+        p->pass_cap = warp_short_cap(p->mode);
         rc = layout_table(p, KERNEL_WARP, threads, nullptr);
         p->pass_cap = asked_cap;
         if (rc != SPDY_OK) return rc;

@@ -49,10 +49,11 @@ constexpr int cluster_cells_per_lane(int threads) { return threads >= 512 ? 16 :
 
 // Longest pass of the 1024-thread kernel whose rows live in global memory (64 registers per thread, 64-bit
 // row addresses).
-constexpr int global_rows_cap_1024(int mode) { return mode == MODE_ARG_PAIR ? 8 : 12; }
+constexpr int global_rows_cap_1024(int mode) { return mode == MODE_ARG_PAIR ? 7 : 11; }
 
-// The warp-per-candidate kernel comes in two builds: passes of up to 8 cells per lane in 64 registers
-// (8 CTAs of 128 threads per SM) and up to long_pass_cap() in 128 registers (4 CTAs).
+// The warp-per-candidate kernel comes in two builds: passes of up to warp_short_cap() cells per lane in 64
+// registers (8 CTAs of 128 threads per SM) and up to long_pass_cap() in 128 registers (4 CTAs).
+constexpr int warp_short_cap(int mode) { return mode == MODE_ARG_PAIR ? 7 : 8; }
 inline bool mode_is_row(int mode) { return mode == MODE_ROW || mode == MODE_ROW2; }
 inline bool mode_is_arg(int mode) { return mode == MODE_ARG || mode == MODE_ARG_PRED || mode == MODE_ARG_PAIR; }
 
