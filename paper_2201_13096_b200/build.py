@@ -83,12 +83,13 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     objdir = os.path.join(OBJ_ROOT, "debug" if debug else "release")
     os.makedirs(objdir, exist_ok=True)
     defines = ["-DSPDY_DEBUG_CHECKS"] if debug else []
+    ptxas_opt = []
     jobs, objects, log = [], [], []
     for src in sources:
         obj = os.path.join(objdir, os.path.basename(src) + ".o")
         objects.append(obj)
         if force or verbose or _stale(obj, [src] + HEADERS):
-            jobs.append([_nvcc(), *NVCC_FLAGS, *defines, *(["-Xptxas", "-v"] if verbose else []), "-c", "-o", obj, src])
+            jobs.append([_nvcc(), *NVCC_FLAGS, *defines, *ptxas_opt, *(["-Xptxas", "-v"] if verbose else []), "-c", "-o", obj, src])
     for src in HOST_SOURCES:
         host_obj = os.path.join(objdir, os.path.basename(src) + ".o")
         objects.append(host_obj)

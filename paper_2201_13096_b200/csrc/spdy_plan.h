@@ -23,7 +23,11 @@ constexpr int kRmax = 24;
 // cell update (packed add + 3-input minimum) unroll passes twice as long: every pass pays for its own
 // 16-byte slot reads (about three data-path wavefronts per pair of slots), so half as many passes take
 // 4 % off the traffic of the unit the kernel is bound by.
+#ifdef SPDY_DEBUG_CHECKS
+constexpr int kRmaxLong = 24;  // the index-checked pass bodies of 48 cells take minutes each to compile
+#else
 constexpr int kRmaxLong = 48;
+#endif
 constexpr int long_pass_cap(int mode) { return mode == 4 /* MODE_ROW2 */ ? kRmaxLong : kRmax; }
 
 // Widest band (cells) for which the plan considers one warp per candidate when left to choose (it then
