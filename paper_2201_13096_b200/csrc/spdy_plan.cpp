@@ -364,7 +364,7 @@ int layout_table(spdy_plan *p, int kind, int threads, double *efficiency)
     int64_t off = 0, max_extent = 32, max_cpl = 1;
     int64_t need_left = 0;
     std::vector<int64_t> need_right(static_cast<size_t>(p->L) + 1, 0);  // cells beyond row l-1's extent that layer l reads
-    double sum_cost = 0.0, sum_span = 0.0;
+    double sum_span = 0.0;
     p->issued_updates = 0;
     std::vector<int> ba, bb;
     std::vector<std::vector<PassPlan>> per_warp;
@@ -385,7 +385,6 @@ int layout_table(spdy_plan *p, int kind, int threads, double *efficiency)
         double total = 0.0, span = 0.0;
         int covered = nb;
         plan_layer_passes(ba, bb, nb, W, R, p->schedule, per_warp, &total, &span, &covered);
-        sum_cost += total;
         sum_span += span * W;
         ld.extent = 32 * covered;
         max_extent = std::max<int64_t>(max_extent, ld.extent);
@@ -444,7 +443,6 @@ int layout_table(spdy_plan *p, int kind, int threads, double *efficiency)
     else p->smem_bytes = 2LL * p->row_stride * 4 + tap_bytes;
     // Needed cell updates per data-path wavefront the busiest warps take: falls with partly overlapping slots,
     // with the passes' own slot reads (short passes pay more of them) and with warps that wait for others.
-    (void)sum_cost;
     if (efficiency) *efficiency = sum_span > 0.0 ? (static_cast<double>(p->distinct_updates) / 32.0) / sum_span : 0.0;
     return SPDY_OK;
 }
@@ -772,7 +770,6 @@ int verify_plan(const spdy_plan *p)
     }
     if (p->kind == KERNEL_CLUSTER) {
         const int C = p->cluster;
-        int64_t prev_width = 1;
         for (int l = 0; l < L; ++l) {
             const LayerDesc &ld = p->layers[l];
             std::vector<int> covered(ld.width, 0);
@@ -797,11 +794,9 @@ int verify_plan(const spdy_plan *p)
                         if (s - tr.a < sd.q0 || s + cells - 1 - tr.a >= sd.q0 + static_cast<int64_t>(sd.win_len)) return SPDY_ERR_INTERNAL;
                     }
                 }
-                (void)prev_width;
             }
             for (int c = 0; c < ld.width; ++c)
                 if (covered[c] != 1) return SPDY_ERR_INTERNAL;
-            prev_width = ld.width;
         }
         return SPDY_OK;
     }
