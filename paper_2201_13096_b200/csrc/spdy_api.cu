@@ -988,7 +988,9 @@ int spdy_solve_batch_simple(const float *errors_dev, const int32_t *times_dev, i
     SPDY_CUDA_TRY(cudaMemcpyAsync(times.data(), times_dev, times.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
     SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
     spdy_plan *plan = nullptr;
-    int rc = spdy_plan_create(&plan, times.data(), L, K, B, device, nullptr);
+    spdy_options opts = {};
+    opts.auto_shape = N >= 300 ? 1 : 0;  // a batch that fills the device needs no launch shapes for small ones
+    int rc = spdy_plan_create(&plan, times.data(), L, K, B, device, &opts);
     if (rc != SPDY_OK) return rc;
     void *ws = nullptr;
     size_t ws_bytes = 0;

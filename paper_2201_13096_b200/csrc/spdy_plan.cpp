@@ -295,7 +295,7 @@ void plan_layer_passes(const std::vector<int> &ba, const std::vector<int> &bb, i
             double lo = 0.0, hi = pass_cost(0, std::min(nb, R)) * 2.0 + 1.0;
             for (int i = 0; i < nb; ++i) lo = std::max(lo, pass_cost(i, i + 1));
             if (cut(hi, nullptr) > P) continue;
-            for (int it = 0; it < 40; ++it) {
+            for (int it = 0; it < 24 && hi - lo > 0.25; ++it) {
                 const double mid = 0.5 * (lo + hi);
                 if (cut(mid, nullptr) <= P) hi = mid;
                 else lo = mid;
@@ -659,11 +659,16 @@ int choose_launch_shape(spdy_plan *p, const spdy_options *opts)
     const int sizes[] = {128, 256, 512, 1024};
     int best_threads = 0;
     double best_score = -1.0;
+    // (scored with passes of one length, which cost a tenth of the levelled partition to lay out and rank the
+    // CTA sizes the same way; the chosen size is laid out for good below)
+    const int wanted_schedule = p->schedule;
     for (int threads : sizes) {
         if (opts && opts->threads && opts->threads != threads) continue;
         if (threads < p->K) continue;  // one thread per choice stages the next layer
         double eff = 0.0;
+        p->schedule = SCHED_UNIFORM;
         int rc = layout_table(p, KERNEL_CTA, threads, &eff);
+        p->schedule = wanted_schedule;
         if (rc != SPDY_OK) return rc;
         if (p->smem_bytes > p->limits.smem_per_block - kStaticSmemReserve) continue;
         const double warps = static_cast<double>(resident_ctas(p, threads, p->smem_bytes) * threads / 32);
