@@ -234,6 +234,34 @@ __device__ __forceinline__ void update_arg_pair(float (&best)[RR], int (&code)[R
 #undef SPDY_PAIR_UPDATE
 }
 
+// The same step from one array of running minima into another.  In place, the 3-input minimum has to land in a
+// fresh register - the compare still needs the old value - and the loop-carried array takes it back with a
+// move per cell and pair; taken two pairs at a time, from `in` to `out` and back, the move disappears.
+template <int RR>
+__device__ __forceinline__ void update_arg_pair_to(const float (&in)[RR], float (&out)[RR], int (&code)[RR], const Src sa,
+                                                   const float ea, const Src sb, const float eb, const int pair_code,
+                                                   const AccessWindow &w)
+{
+    const unsigned long long ea2 = splat2(ea), eb2 = splat2(eb);
+#pragma unroll
+    for (int j = 0; j + 1 < RR; j += 2) {
+        float a0 = sa.at(j, w), a1 = sa.at(j + 1, w);
+        float b0 = sb.at(j, w), b1 = sb.at(j + 1, w);
+        add2_rn(a0, a1, ea2);
+        add2_rn(b0, b1, eb2);
+        out[j] = min3(in[j], a0, b0);
+        code[j] = (out[j] < in[j]) ? pair_code : code[j];
+        out[j + 1] = min3(in[j + 1], a1, b1);
+        code[j + 1] = (out[j + 1] < in[j + 1]) ? pair_code : code[j + 1];
+    }
+    if (RR & 1) {
+        const float a0 = __fadd_rn(sa.at(RR - 1, w), ea);
+        const float b0 = __fadd_rn(sb.at(RR - 1, w), eb);
+        out[RR - 1] = min3(in[RR - 1], a0, b0);
+        code[RR - 1] = (out[RR - 1] < in[RR - 1]) ? pair_code : code[RR - 1];
+    }
+}
+
 // Codes of update_arg_pair -> slot indices, once per pass.  A cell whose code names a pair (odd) won with
 // m = min(v0, v1) of that pair and nothing after it was smaller, so best still holds that m: the winner is
 // k0 if v0 - the same fp32 add of the same operands, hence the same bits - equals best, else k1 (a tie
@@ -305,7 +333,8 @@ __device__ __forceinline__ void update_arg_pred(float (&best)[RR], float (&idxf)
 //
 // With STORE_TABLE false (row-value table only) the pass leaves the table alone: the caller copies the whole
 // row from shared memory to the table with one bulk copy per layer.
-template <int RR, int MODE, bool MASKED, bool STORE_TABLE = true>
+// ROOMY: the build has 128 registers per thread (see update_arg_pair_to).
+template <int RR, int MODE, bool MASKED, bool STORE_TABLE = true, bool ROOMY = false>
 __device__ __forceinline__ void process_span(const float *prev, float *cur, const int2 *__restrict__ taps,
                                              const unsigned krange, const unsigned long long *__restrict__ mask,
                                              const int MW, const int s, const int lane, void *table_row,
@@ -418,6 +447,21 @@ __device__ __forceinline__ void process_span(const float *prev, float *cur, cons
                 update_arg<RR>(best, code, make_src(prev, first, tp.x), __int_as_float(tp.y), 2 * k, w);
                 ++k;
             }
+            // Two pairs per trip, the running minima alternating between `best` and `other` (see
+            // update_arg_pair_to) - for passes of up to 20 cells per lane: beyond, the third register array no
+            // longer fits the 128 registers of a thread.
+            if constexpr (ROOMY && RR <= 20) {
+                float other[RR];
+#pragma unroll 1
+                for (; k + 3 < k_hi; k += 4) {
+                    const int4 t = *reinterpret_cast<const int4 *>(taps + k);
+                    const int4 t2 = *reinterpret_cast<const int4 *>(taps + k + 2);
+                    update_arg_pair_to<RR>(best, other, code, make_src(prev, first, t.x), __int_as_float(t.y),
+                                           make_src(prev, first, t.z), __int_as_float(t.w), 2 * k + 1, w);
+                    update_arg_pair_to<RR>(other, best, code, make_src(prev, first, t2.x), __int_as_float(t2.y),
+                                           make_src(prev, first, t2.z), __int_as_float(t2.w), 2 * k + 5, w);
+                }
+            }
 #pragma unroll 1
             for (; k + 1 < k_hi; k += 2) {
                 const int4 t = *reinterpret_cast<const int4 *>(taps + k);
@@ -484,7 +528,7 @@ __device__ __forceinline__ void process_span(const float *prev, float *cur, cons
 }
 
 // Runs the pass `pd` with the unrolled body for its cells-per-lane count (1..RCAP).
-template <int MODE, int RCAP, bool MASKED, bool STORE_TABLE = true>
+template <int MODE, int RCAP, bool MASKED, bool STORE_TABLE = true, bool ROOMY = false>
 __device__ __forceinline__ void run_pass(const int cpl, const float *prev, float *cur, const int2 *taps,
                                          const unsigned krange, const unsigned long long *mask, const int MW,
                                          const int s, const int lane, void *table_row, const int limit,
@@ -494,8 +538,8 @@ __device__ __forceinline__ void run_pass(const int cpl, const float *prev, float
 #define SPDY_CASE(RR)                                                                                          \
     case RR:                                                                                                   \
         if constexpr (RR <= kRmaxLong && RR <= RCAP)                                                           \
-            process_span<RR, MODE, MASKED, STORE_TABLE>(prev, cur, taps, krange, mask, MW, s, lane, table_row, \
-                                                        limit, w);                                             \
+            process_span<RR, MODE, MASKED, STORE_TABLE, ROOMY>(prev, cur, taps, krange, mask, MW, s, lane,     \
+                                                               table_row, limit, w);                           \
         break;
         SPDY_CASE(1) SPDY_CASE(2) SPDY_CASE(3) SPDY_CASE(4) SPDY_CASE(5) SPDY_CASE(6)
         SPDY_CASE(7) SPDY_CASE(8) SPDY_CASE(9) SPDY_CASE(10) SPDY_CASE(11) SPDY_CASE(12)
@@ -565,6 +609,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
 #else
     constexpr bool BULK = ROWFMT && !GROWS;  // rows in shared memory, row-value table: bulk copy per layer
 #endif
+    constexpr bool ROOMY = NT * MINB <= 512 && !GROWS;  // 128 registers per thread
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float *rows;
     int2 *tap_buf;
@@ -634,7 +679,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
             // (64 registers per thread: no room to hold the next pass's descriptor across a pass)
             for (int p = p0; p < p1; ++p) {
                 const int2 pd = __ldg(reinterpret_cast<const int2 *>(args.passes + p));
-                run_pass<MODE, RCAP, false, !BULK>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+                run_pass<MODE, RCAP, false, !BULK, ROOMY>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
                                             args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
             }
         } else {
@@ -643,7 +688,7 @@ __global__ void __launch_bounds__(NT, MINB) spdy_forward_kernel(const FwdArgs ar
             for (int p = p0; p < p1; ++p) {
                 const int2 pd = pd_next;
                 if (p + 1 < p1) pd_next = __ldg(reinterpret_cast<const int2 *>(args.passes + p + 1));
-                run_pass<MODE, RCAP, false, !BULK>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+                run_pass<MODE, RCAP, false, !BULK, ROOMY>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
                                             args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
             }
         }
@@ -717,6 +762,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, MINB) spdy_forward_warp_ke
 #else
     constexpr bool BULK = ROWFMT;  // row-value table: one bulk copy per layer and warp (see bulk_copy_row_to_table)
 #endif
+    constexpr bool ROOMY = MINB <= 4;  // 128 registers per thread
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -774,7 +820,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, MINB) spdy_forward_warp_ke
         for (int p = p0; p < p1; ++p) {
             const int2 pd = pd_next;
             if (p + 1 < p1) pd_next = __ldg(reinterpret_cast<const int2 *>(args.passes + p + 1));
-            run_pass<MODE, RCAP, false, !BULK>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
+            run_pass<MODE, RCAP, false, !BULK, ROOMY>(static_cast<unsigned>(pd.y) >> 24, prev, cur, taps, static_cast<unsigned>(pd.y),
                                         args.pass_masks + static_cast<size_t>(p) * MW, MW, pd.x, lane, row_base, 0, w);
         }
         for (int i = lane; i < ld.fill; i += 32) cur[ld.extent + i] = INF;
