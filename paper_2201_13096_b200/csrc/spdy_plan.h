@@ -14,7 +14,7 @@
 
 namespace spdy {
 
-constexpr int kLibraryVersion = 2003;
+constexpr int kLibraryVersion = 2004;
 
 // Most band cells one lane owns in one warp pass; the kernels unroll passes of 1..kRmax cells per lane.
 constexpr int kRmax = 24;
