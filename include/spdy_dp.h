@@ -238,7 +238,8 @@ int spdy_solve_batch(const spdy_plan *plan, const float *errors_dev, int64_t N,
  * two host-buffer solves at the same time.  An error table larger than one wave of CTAs is uploaded in
  * a few chunks on a second, plan-owned stream (ordered after the work already queued on `cuda_stream`),
  * each chunk's kernels waiting only for their own chunk, so that with pinned host memory the upload
- * hides behind the kernels.
+ * hides behind the kernels; chunk sizes follow the upload and solving rates the previous call on the plan
+ * measured, and a table whose upload is cheaper than a chunk boundary goes up in one piece.
  */
 int spdy_solve_batch_host(spdy_plan *plan, const float *errors_host, int64_t N,
                           uint8_t *profile_host, float *cost_host, int32_t *time_used_host,

@@ -72,6 +72,12 @@ struct spdy::DeviceSide {
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t entry_event = nullptr;
     std::vector<cudaEvent_t> copy_events;
+    // how fast the first chunk went up and how fast it was solved, timed in every chunked call: the ratio
+    // sets how much larger than its predecessor a chunk may be for its upload to hide behind the kernels
+    cudaEvent_t probe[4] = {nullptr, nullptr, nullptr, nullptr};
+    double chunk_growth = 6.0;
+    double upload_ms_per_byte = 0.0;  // 0 = not measured yet
+    double first_wave_ms = 0.0;
     // staging for the host-buffer entry points
     unsigned char *arena = nullptr;
     size_t arena_bytes = 0;
@@ -433,6 +439,8 @@ void hook_release(spdy_plan *p)
         for (cudaEvent_t e : d->events) cudaEventDestroy(e);
         for (cudaEvent_t e : d->copy_events) cudaEventDestroy(e);
         if (d->entry_event) cudaEventDestroy(d->entry_event);
+        for (cudaEvent_t e : d->probe)
+            if (e) cudaEventDestroy(e);
         if (d->copy_stream) cudaStreamDestroy(d->copy_stream);
     }
     delete d;
@@ -675,10 +683,10 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
     const size_t off_cost = off_profile + round_up(static_cast<size_t>(N) * plan->L, 256);
     const size_t off_time = off_cost + round_up(static_cast<size_t>(N) * 4, 256);
     const size_t off_ws = off_time + round_up(static_cast<size_t>(N) * 4, 256);
-    // Cap the table at 8 GiB; larger batches run as waves.
+    // Cap the table at 16 GiB; larger batches run as waves.
     const size_t ws_full = plan->feasible ? spdy_workspace_bytes(plan, N) : 0;
     const size_t ws_unit = plan->feasible ? spdy_workspace_bytes(plan, 1) : 0;
-    const size_t ws_cap = std::max<size_t>(ws_unit, static_cast<size_t>(8) << 30);
+    const size_t ws_cap = std::max<size_t>(ws_unit, static_cast<size_t>(16) << 30);
     const size_t ws_bytes = std::min(ws_full, ws_cap) / std::max<size_t>(ws_unit, 1) * ws_unit;
     const size_t total = off_ws + ws_bytes;
     if (total > d->arena_bytes) {
@@ -709,23 +717,35 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
     // Everything from the first queued copy on runs inside `enqueue`: whatever makes it stop early, the
     // copies already queued still read the caller's host buffer, so every exit waits for both streams
     // before the error goes back to the caller (who may free or reuse the buffer on seeing it).
+    bool chunked = false;
+    size_t first_chunk_bytes = 1;
     auto enqueue = [&]() -> int {
-        // An error table goes up in chunks of growing size (one full wave of CTAs first, then six times
-        // the previous chunk) on a second stream, so that every upload but the first hides behind the
-        // kernels of the chunk before it; an upload takes about a seventh of the time its candidates take
-        // to solve.  Every chunk boundary costs a launch tail (and a walk back, unless one serves all), so
-        // chunks are few - one wave, then the rest, measured best at the BERT-base shape - and coefficient
-        // input (K times smaller) goes up in one piece.
+        // An error table goes up in chunks of growing size on a second stream, so that every upload but the
+        // first hides behind the kernels of the chunk before it.  The first chunk is one full wave of CTAs; each
+        // further one may be larger than its predecessor by the ratio of solving time to upload time per
+        // candidate, which the previous call on this plan measured on its first chunk (about 6 with a fast
+        // host link, 2 to 3 with a slow one; 6 until measured).  Every chunk boundary costs a launch tail (and a
+        // walk back, unless one serves all), so a remainder not much larger than the next chunk goes with it,
+        // and coefficient input (K times smaller) goes up in one piece.
         const int64_t per_cand = static_cast<int64_t>(plan->L) * (coeffs ? 1 : plan->K);
         std::vector<int64_t> bounds(1, 0);
         {
             const int64_t per_cta = shape->kind == KERNEL_WARP ? shape->threads / 32 : 1;
-            int64_t size = std::max<int64_t>(1, static_cast<int64_t>(shape->ctas_per_sm) * shape->limits.sm_count * per_cta /
-                                                    std::max(1, shape->cluster));
-            if (coeffs) size = N;
+            double size = static_cast<double>(std::max<int64_t>(1, static_cast<int64_t>(shape->ctas_per_sm) * shape->limits.sm_count *
+                                                                       per_cta / std::max(1, shape->cluster)));
+            if (coeffs) size = static_cast<double>(N);
+            // A chunk boundary costs about half a wave of CTAs (the tail of one launch and the ramp of the next);
+            // chunking saves at most the upload time of everything behind the first chunk.  Where a wave is long
+            // and the table small (BERT-large shape: 3.8 ms against 1.3 ms) one piece is the better deal.
+            if (d->upload_ms_per_byte > 0.0 && static_cast<double>(N) > size) {
+                const double saved = (static_cast<double>(N) - size) * static_cast<double>(per_cand) * 4.0 * d->upload_ms_per_byte;
+                if (saved < 0.5 * d->first_wave_ms) size = static_cast<double>(N);
+            }
             while (bounds.back() < N) {
-                bounds.push_back(std::min<int64_t>(N, bounds.back() + size));
-                size *= 6;
+                const int64_t left = N - bounds.back();
+                const int64_t take = static_cast<double>(left) <= 1.35 * size ? left : static_cast<int64_t>(size);
+                bounds.push_back(bounds.back() + std::max<int64_t>(1, take));
+                size *= d->chunk_growth;
             }
         }
         const size_t chunks = bounds.size() - 1;
@@ -740,11 +760,15 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
             // Work already queued on the caller's stream may still read the staging buffer.
             SPDY_CUDA_TRY(cudaEventRecord(d->entry_event, stream));
             SPDY_CUDA_TRY(cudaStreamWaitEvent(d->copy_stream, d->entry_event, 0));
+            for (cudaEvent_t &e : d->probe)
+                if (!e) SPDY_CUDA_TRY(cudaEventCreate(&e));
             for (size_t c = 0; c < chunks; ++c) {
                 const int64_t first = bounds[c], count = bounds[c + 1] - bounds[c];
+                if (c == 0) SPDY_CUDA_TRY(cudaEventRecord(d->probe[0], d->copy_stream));
                 SPDY_CUDA_TRY(cudaMemcpyAsync(d_err + first * per_cand, errors_host + first * per_cand,
                                               static_cast<size_t>(count * per_cand) * sizeof(float),
                                               cudaMemcpyHostToDevice, d->copy_stream));
+                if (c == 0) SPDY_CUDA_TRY(cudaEventRecord(d->probe[1], d->copy_stream));
                 SPDY_CUDA_TRY(cudaEventRecord(d->copy_events[c], d->copy_stream));
             }
         } else {
@@ -759,6 +783,7 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
         for (size_t c = 0; c < chunks; ++c) {
             const int64_t first = bounds[c], count = bounds[c + 1] - bounds[c];
             if (chunks > 1) SPDY_CUDA_TRY(cudaStreamWaitEvent(stream, d->copy_events[c], 0));
+            if (chunks > 1 && c <= 1) SPDY_CUDA_TRY(cudaEventRecord(d->probe[2 + c], stream));  // around chunk 0's kernels
             const float *in = d_err + first * per_cand;
             if (one_walk_back)
                 lrc = solve_impl(plan, shape, coeffs ? nullptr : in, coeffs ? in : nullptr, count, d_profile + first * plan->L,
@@ -777,6 +802,8 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
         SPDY_CUDA_TRY(cudaMemcpyAsync(profile_host, d_profile, static_cast<size_t>(N) * plan->L, cudaMemcpyDeviceToHost, stream));
         SPDY_CUDA_TRY(cudaMemcpyAsync(cost_host, d_cost, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
         SPDY_CUDA_TRY(cudaMemcpyAsync(time_used_host, d_time, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, stream));
+        chunked = chunks > 1;
+        first_chunk_bytes = static_cast<size_t>(bounds[1] * per_cand) * sizeof(float);
         return SPDY_OK;
     };
     rc = enqueue();
@@ -786,6 +813,17 @@ int solve_host_impl(spdy_plan *plan, const float *errors_host, bool coeffs, int6
         return rc;
     }
     SPDY_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (chunked) {
+        // (probe[3] was recorded after chunk 1's upload had arrived, i.e. it may include waiting for it: the
+        // ratio then comes out too large by at most that wait, which the factor 0.85 and the bounds absorb)
+        float up_ms = 0.f, solve_ms = 0.f;
+        if (cudaEventElapsedTime(&up_ms, d->probe[0], d->probe[1]) == cudaSuccess &&
+            cudaEventElapsedTime(&solve_ms, d->probe[2], d->probe[3]) == cudaSuccess && up_ms > 0.f && solve_ms > 0.f) {
+            d->chunk_growth = std::min(8.0, std::max(1.5, 0.85 * static_cast<double>(solve_ms) / up_ms));
+            d->upload_ms_per_byte = static_cast<double>(up_ms) / static_cast<double>(first_chunk_bytes);
+            d->first_wave_ms = solve_ms;
+        }
+    }
     return SPDY_OK;
 }
 
