@@ -57,7 +57,8 @@ typedef enum spdy_status {
  *   per cell, merges choices of equal time unconditionally, and runs about 1.3x faster; the table is
  *   4 bytes per cell.
  *   ARG_U8 keeps Algorithm 1's matrix P (the winning choice index), one byte per cell, at the
- *   price of a compare and two selects per cell update.  Use it when workspace is scarce.
+ *   price of a compare and a select (taken over pairs of choices) per cell update on top of add and
+ *   minimum: about 1.3x the forward time of ROW_F32.  Use it when workspace is scarce.
  *   Equal-time choices can be merged here only for candidates whose errors do not fall with the
  *   choice index inside any group of equal-time choices (always true for Eq. 4's errors with
  *   non-negative coefficients); a small kernel tests that per candidate, and the others run with one
@@ -88,7 +89,8 @@ typedef struct spdy_options {
                               identical results, for measurement: 1 compare+select (ARG_U8),
                               2 compare+predicated moves (ARG_U8), 3 fp32 minimum (ROW_F32),
                               4 packed adds + 3-input minimum over slot pairs (ROW_F32),
-                              5 3-input minimum over slot pairs, index resolved from the outcome (ARG_U8) */
+                              5 3-input minimum over slot pairs, the winner inside a pair settled once per
+                              warp pass (ARG_U8) */
     int32_t rows_in_global; /* 1: keep the two dynamic-program rows in the workspace (global memory) rather than
                               in shared memory and read them through L1.  Chosen automatically when two rows
                               do not fit one CTA's shared memory (B of about 10^5 buckets and more); any width
