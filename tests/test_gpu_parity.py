@@ -667,3 +667,40 @@ def test_small_batches_pick_their_launch_shape_by_themselves(fmt):
     assert_same(binding.solve_batch_host(plan, wl.errors[:160]), tuple(x[:160] for x in ref))
     plan.close()
     pinned.close()
+
+
+def test_plans_solved_from_two_host_threads_at_once():
+    """The library keeps no global state: two host threads, each with its own plan, stream and buffers, solve
+    different problems at the same time, again and again, and both stay bit-exact."""
+    import threading
+
+    import torch
+
+    jobs = []
+    for cfg, n, fmt in ((2, 40, binding.SPDY_TABLE_ROW_F32), (1, 60, binding.SPDY_TABLE_ARG_U8)):
+        wl = W.make_workload(cfg, N=n)
+        jobs.append((wl, fmt, oracle.solve_batch(wl.errors, wl.times, wl.B, threads=CORES)))
+    failures = []
+
+    def worker(wl, fmt, ref):
+        try:
+            stream = torch.cuda.Stream()
+            plan = binding.Plan(wl.times, wl.B, device=0, table_format=fmt)
+            errors = torch.from_numpy(wl.errors).cuda()
+            torch.cuda.synchronize()
+            for _ in range(12):
+                p, c, t = binding.solve_batch(plan, errors, stream=stream)
+                stream.synchronize()
+                plan.check_status(stream)
+                assert_same((p.cpu().numpy(), c.cpu().numpy(), t.cpu().numpy()), ref)
+                assert_same(binding.solve_batch_host(plan, wl.errors, stream=stream), ref)
+            plan.close()
+        except BaseException as exc:  # reported by the main thread
+            failures.append(exc)
+
+    threads = [threading.Thread(target=worker, args=job) for job in jobs]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    assert not failures, failures

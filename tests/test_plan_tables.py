@@ -274,6 +274,23 @@ def test_small_batches_get_their_own_launch_shapes():
         assert binding.Plan(wl.times, wl.B, device=-1, **pinned).info["alternates"] == 0
 
 
+def test_launch_shape_by_batch_size():
+    """Which table set a batch runs on: the largest cluster that still gives every CTA an SM, a 512-thread CTA
+    while every candidate can have an SM to itself, the main shape from there on - and the main shape whenever
+    the workspace is too small for the shape picked."""
+    wl = W.make_workload(2, N=1)
+    plan = binding.Plan(wl.times, wl.B, device=-1)
+    shape = {n: plan.shape_for_batch(n) for n in (1, 18, 19, 37, 38, 74, 75, 148, 149, 295, 296, 4096)}
+    assert [shape[n]["cluster"] for n in (1, 18, 19, 37, 38, 74)] == [8, 8, 4, 4, 2, 2]
+    assert all(shape[n]["kernel_kind"] == 2 for n in (1, 18, 19, 37, 38, 74))
+    assert shape[75]["kernel_kind"] == 0 and shape[75]["threads"] == 512 and shape[148]["threads"] == 512
+    for n in (149, 295, 296, 4096):
+        assert shape[n]["which"] == 0 and shape[n]["threads"] == plan.info["threads"]
+    tight = binding.Plan(wl.times, wl.B, device=-1, auto_shape=1).workspace_bytes(2)
+    assert plan.shape_for_batch(7, tight)["which"] == 0
+    assert binding.library().spdy_plan_shape_for_batch(None, 5, 0) == -1
+
+
 def test_narrow_rows_take_the_warp_kernel():
     wl = W.make_workload(4, N=1, B=1000)
     info = binding.Plan(wl.times, wl.B, device=-1).info
