@@ -117,21 +117,30 @@ def spilling_kernels(log: str) -> list:
 
 
 def build_all(force: bool = False) -> None:
-    """All three libraries; a forced build also checks that no kernel of the product library spills."""
-    if force:
-        import contextlib
-        import io
+    """All three libraries, the product and the debug library side by side; a forced build also checks that no
+    kernel of the product library spills."""
+    log = []
 
-        buf = io.StringIO()
-        with contextlib.redirect_stdout(buf):
-            build(force=True, verbose=True)
-        bad = spilling_kernels(buf.getvalue())
-        if bad:
-            raise RuntimeError("kernels with register spills: " + ", ".join(bad))
-    else:
-        build()
-    build(force=force, debug=True)
+    def product():
+        if force:
+            import contextlib
+            import io
+
+            buf = io.StringIO()
+            with contextlib.redirect_stdout(buf):
+                build(force=True, verbose=True)
+            log.append(buf.getvalue())
+        else:
+            build()
+
+    with ThreadPoolExecutor(max_workers=2) as pool:
+        jobs = [pool.submit(product), pool.submit(build, force, False, True)]
+        for job in jobs:
+            job.result()
     build_host(force=force)
+    bad = spilling_kernels("".join(log))
+    if bad:
+        raise RuntimeError("kernels with register spills: " + ", ".join(bad))
 
 
 if __name__ == "__main__":
